@@ -1,0 +1,490 @@
+#!/usr/bin/env python
+"""Benchmark of the GAC hot path (stats + projection + state refresh).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+
+One "step" is one pass of the whole path over one synthetic gradient list:
+gac_stats (fused <g,d>, <g,g>, <d,d>, cosine, regime, gains) followed by
+gac_project (in-place rank-one update, stored direction refreshed), in the
+projection regime -- the regime that moves the most bytes.
+
+Timing: CUDA events on the launching stream around the two calls of every
+step, summed over the K timed steps; between steps a FRESH gradient with the
+configured cosine to the stored direction is written into g (as the backward
+pass of a training loop would), outside the timed events; that write also
+evicts the 126 MB L2.  Prints one JSON line.
+"""
+from __future__ import annotations
+
+import argparse
+import hashlib
+import json
+import math
+import os
+import statistics
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import torch  # noqa: E402
+
+from paper_2603_01501_b200 import synth  # noqa: E402
+
+METRIC = "GAC stats+projection params/s"
+UNIT = "params/s"
+FORCE = dict(c_low=0.05, c_high=2.0)   # legal thresholds that keep every step in the projection regime
+NOMINAL_HBM_GBS = 8000.0
+
+
+# ----------------------------------------------------------------- utilities
+
+def measured_hbm_peak():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(p) as fh:
+            return float(json.load(fh)["hbm_gbs"]), "measured"
+    except Exception:
+        return 6650.0, "fallback"
+
+
+def bytes_per_param(g_dtype) -> int:
+    sg = 2 if g_dtype == torch.bfloat16 else 4
+    return sg + 4
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons through NVML (read-only) while the
+    timed region runs."""
+
+    def __init__(self, index: int, period_s: float = 0.1):
+        self.index, self.period = index, period_s
+        self.samples, self.reasons, self.max_mhz = [], set(), None
+        self._stop = threading.Event()
+        self._thr = None
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM)
+        except Exception:
+            self.nv = None
+
+    def _loop(self):
+        nv = self.nv
+        names = {"hw_slowdown": getattr(nv, "nvmlClocksEventReasonHwSlowdown", 0x8),
+                 "hw_thermal_slowdown": getattr(nv, "nvmlClocksEventReasonHwThermalSlowdown", 0x40),
+                 "sw_thermal_slowdown": getattr(nv, "nvmlClocksEventReasonSwThermalSlowdown", 0x20),
+                 "sw_power_cap": getattr(nv, "nvmlClocksEventReasonSwPowerCap", 0x4)}
+        while not self._stop.is_set():
+            try:
+                self.samples.append(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM))
+                try:
+                    mask = nv.nvmlDeviceGetCurrentClocksEventReasons(self.h)
+                except Exception:
+                    mask = nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h)
+                for k, bit in names.items():
+                    if mask & bit:
+                        self.reasons.add(k)
+            except Exception:
+                pass
+            self._stop.wait(self.period)
+
+    def __enter__(self):
+        if self.nv is not None:
+            self._thr = threading.Thread(target=self._loop, daemon=True)
+            self._thr.start()
+        return self
+
+    def __exit__(self, *a):
+        self._stop.set()
+        if self._thr:
+            self._thr.join()
+
+    def summary(self):
+        if not self.samples:
+            return {"sm_mhz": None, "sm_max_mhz": self.max_mhz, "reasons": ["nvml unavailable"]}
+        return {"sm_mhz": statistics.median(self.samples), "sm_max_mhz": self.max_mhz,
+                "reasons": sorted(self.reasons), "samples": len(self.samples)}
+
+
+def nvml_index(local_rank: int) -> int:
+    vis = os.environ.get("CUDA_VISIBLE_DEVICES")
+    if vis:
+        try:
+            return int(vis.split(",")[local_rank])
+        except Exception:
+            return local_rank
+    return local_rank
+
+
+def recorded_traffic(kernel: str):
+    """DRAM bytes per parameter of `kernel` from the committed ncu capture, or
+    None when the kernel source changed since the capture."""
+    try:
+        with open(os.path.join(ROOT, "profiles", "traffic.json")) as fh:
+            rec = json.load(fh)
+        src = os.path.join(ROOT, "paper_2603_01501_b200", "csrc", "gac.cu")
+        if hashlib.sha256(open(src, "rb").read()).hexdigest() != rec["source_sha256"]:
+            return None
+        return rec["kernels"][kernel]
+    except Exception:
+        return None
+
+
+# --------------------------------------------------------------- GPU workload
+
+class Workload:
+    def __init__(self, name: str, device, world: int):
+        from paper_2603_01501_b200 import binding as gb
+        self.gb = gb
+        dims_key, self.g_dtype, self.rho, self.config_id = synth.WORKLOADS[name]
+        self.name, self.device, self.world = name, device, world
+        self.shapes = synth.decoder_tensor_list(synth.DIMS[dims_key])
+        self.params = synth.list_numel(self.shapes)
+        self.sigma = synth.per_tensor_scales(self.config_id, len(self.shapes))
+        self.g, self.d = synth.gradient_list(self.shapes, self.rho, self.config_id, self.g_dtype, device)
+        self.scratch = torch.empty(max(n for _, n in self.shapes), dtype=torch.float32, device=device)
+        self.gen = torch.Generator(device=device)
+        self.gen.manual_seed(12345 + self.config_id)
+        self.ctx = gb.gac_init(self.g, self.d, gb.HParams(**FORCE))
+        self.step_no = 1      # the stored direction already holds g_{t-1}
+        self.sums = torch.zeros(3, dtype=torch.float64, device=device) if world > 1 else None
+
+    def refresh(self):
+        synth.refresh_gradient_list(self.g, self.d, self.sigma, self.rho, self.gen, self.scratch)
+
+    def step(self, ev=None):
+        """stats + project on the current stream; ev = three CUDA events or None."""
+        gb = self.gb
+        self.step_no += 1
+        if ev:
+            ev[0].record()
+        if self.world > 1:
+            # sharded form: local sums, ONE all-reduce of three numbers, same decision on every rank
+            gb.gac_stats_partial(self.ctx, self.step_no, self.sums)
+            torch.distributed.all_reduce(self.sums)
+            gb.gac_decide(self.ctx, self.sums, fetch=False)
+        else:
+            gb.gac_stats(self.ctx, self.step_no, fetch=False)
+        if ev:
+            ev[1].record()
+        gb.gac_project(self.ctx)
+        if ev:
+            ev[2].record()
+
+    def close(self):
+        self.gb.gac_free(self.ctx)
+        self.g = self.d = self.scratch = None
+        torch.cuda.empty_cache()
+
+
+def time_steps(wl: Workload, steps: int, warmup: int, sampler=None):
+    """Returns (stats_ms list, project_ms list) of the timed steps."""
+    for _ in range(warmup):
+        wl.refresh()
+        wl.step()
+    torch.cuda.synchronize()
+    evs = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(steps)]
+    if wl.world > 1:
+        torch.distributed.barrier()
+    torch.cuda.synchronize()
+    ctxmgr = sampler if sampler is not None else _Null()
+    with ctxmgr:
+        for i in range(steps):
+            wl.refresh()
+            wl.step(evs[i])
+        torch.cuda.synchronize()
+    if wl.world > 1:
+        torch.distributed.barrier()
+    s_ms = [e[0].elapsed_time(e[1]) for e in evs]
+    p_ms = [e[1].elapsed_time(e[2]) for e in evs]
+    return s_ms, p_ms
+
+
+class _Null:
+    def __enter__(self):
+        return self
+
+    def __exit__(self, *a):
+        return False
+
+
+def check_regime(wl: Workload):
+    """One extra (untimed) step that fetches the decision: the timed steps must
+    have been projection steps with the configured cosine."""
+    wl.refresh()
+    gb = wl.gb
+    wl.step_no += 1
+    if wl.world > 1:
+        gb.gac_stats_partial(wl.ctx, wl.step_no, wl.sums)
+        torch.distributed.all_reduce(wl.sums)
+        res = gb.gac_decide(wl.ctx, wl.sums)
+    else:
+        res = gb.gac_stats(wl.ctx, wl.step_no)
+    gb.gac_project(wl.ctx)
+    torch.cuda.synchronize()
+    return res
+
+
+def time_e2e(wl: Workload, steps: int, warmup: int):
+    """Same step through the C ABI with HOST buffers: every step copies the
+    gradient list from pinned host memory to the device, runs stats + project,
+    and copies the updated gradient list and the decision record back.  Wall
+    clock around the whole step, device idle on both sides."""
+    gb = wl.gb
+    pinned = True
+    try:
+        host_g = [torch.empty(t.shape, dtype=t.dtype, pin_memory=True) for t in wl.g]
+    except RuntimeError:
+        pinned = False
+        host_g = [torch.empty(t.shape, dtype=t.dtype) for t in wl.g]
+    h2d = sum(h.numel() * h.element_size() for h in host_g)
+    d2h = h2d + 72      # g' and the 72-byte decision record
+    times = []
+    for i in range(warmup + steps):
+        wl.refresh()                       # next gradient, staged on the host (untimed)
+        for h, t in zip(host_g, wl.g):
+            h.copy_(t)
+            t.zero_()
+        torch.cuda.synchronize()
+        t0 = time.perf_counter()
+        for h, t in zip(host_g, wl.g):
+            t.copy_(h, non_blocking=True)
+        wl.step_no += 1
+        gb.gac_stats(wl.ctx, wl.step_no, fetch=False)
+        gb.gac_project(wl.ctx, fetch=True)          # reads the decision record back
+        for h, t in zip(host_g, wl.g):
+            h.copy_(t, non_blocking=True)
+        torch.cuda.synchronize()
+        if i >= warmup:
+            times.append((time.perf_counter() - t0) * 1e3)
+    ms = sum(times) / len(times)
+    return {"value": wl.params * wl.world / (ms * 1e-3), "unit": UNIT, "ms_per_step": ms,
+            "steps": steps, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+            "pinned": pinned}
+
+
+# ------------------------------------------------------------- CPU baseline
+
+def oracle_sample(name: str, target_elems: int):
+    """A prefix of the workload's tensor list (whole tensors, the last one cut),
+    generated on the CPU with the list's recipe."""
+    dims_key, g_dtype, rho, config_id = synth.WORKLOADS[name]
+    shapes = synth.decoder_tensor_list(synth.DIMS[dims_key])
+    # skip the embedding so that the sample holds the per-layer mix of small and large tensors
+    sig = synth.per_tensor_scales(config_id, len(shapes))
+    gs, ds, total, used = [], [], 0, 0
+    for i in range(1, len(shapes)):
+        n = min(shapes[i][1], target_elems - total)
+        if n <= 0:
+            break
+        g, d = synth.gaussian_tensor_pair(n, sig[i], rho, config_id, i, g_dtype, "cpu")
+        gs.append(g)
+        ds.append(d)
+        total += n
+        used += 1
+    return gs, ds, total, used
+
+
+def time_oracle(name: str, target_elems: int, steps: int, warmup: int):
+    from oracle import gac_oracle as orc
+    threads = len(os.sched_getaffinity(0)) if hasattr(os, "sched_getaffinity") else os.cpu_count()
+    gs, ds, total, used = oracle_sample(name, target_elems)
+    hp = orc.HParams(**FORCE)
+    times = []
+    for i in range(warmup + steps):
+        g = [t.clone() for t in gs]
+        d = [t.clone() for t in ds]
+        t0 = time.perf_counter()
+        orc.step(g, d, hp, threads=threads)
+        dt = time.perf_counter() - t0
+        if i >= warmup:
+            times.append(dt)
+    sec = sum(times) / len(times)
+    return {"value": total / sec, "unit": UNIT, "cores": threads, "kind": "oracle",
+            "sample": f"tensors 1..{used} of the {name} list ({total} params), stats+project, "
+                      f"{steps} timed passes of {sec:.2f} s", "seconds_per_pass": sec}
+
+
+def run_reference(args):
+    """The CPU oracle as it stands, on the host cores, on the same workload
+    definition (a bounded sample of it per step)."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return 0
+    name = args.workload
+    # calibrate so that warmup+steps passes end within about two minutes
+    probe = time_oracle(name, 8_000_000, 1, 0)
+    budget_s = 100.0 / max(1, args.steps + args.warmup)
+    target = int(min(2_000_000_000, max(8_000_000, probe["value"] * budget_s)))
+    cb = time_oracle(name, target, args.steps, args.warmup)
+    dims_key, g_dtype, rho, config_id = synth.WORKLOADS[name]
+    line = {"impl": "reference", "metric": METRIC, "value": cb["value"], "unit": UNIT,
+            "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup,
+            "ms_per_step": cb["seconds_per_pass"] * 1e3, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": workload_config(name, None),
+            "cpu_baseline": {k: cb[k] for k in ("value", "unit", "cores", "kind", "sample")},
+            "e2e": {"value": cb["value"], "unit": UNIT, "h2d_bytes_per_step": 0,
+                    "d2h_bytes_per_step": 0}}
+    print(json.dumps(line))
+    return 0
+
+
+def workload_config(name: str, wl):
+    dims_key, g_dtype, rho, config_id = synth.WORKLOADS[name]
+    shapes = synth.decoder_tensor_list(synth.DIMS[dims_key])
+    return {"workload": f"{name}: {dims_key} decoder-shaped gradient list, "
+                        f"{'bf16' if g_dtype == torch.bfloat16 else 'f32'} g / f32 d, target cosine {rho}, "
+                        f"projection regime forced with c_low=0.05 c_high=2.0",
+            "params_per_gpu": synth.list_numel(shapes), "tensors": len(shapes),
+            "bytes_per_param": 3 * bytes_per_param(g_dtype),
+            "l2": "inputs larger than L2; a fresh gradient is written between timed steps",
+            "timing": "per-step CUDA events around gac_stats+gac_project, summed over the timed steps"}
+
+
+# ------------------------------------------------------------------- driver
+
+def summarize(wl: Workload, s_ms, p_ms, peak, peak_kind):
+    bpp = bytes_per_param(wl.g_dtype)
+    s_avg, p_avg = sum(s_ms) / len(s_ms), sum(p_ms) / len(p_ms)
+    step_ms = s_avg + p_avg
+    proj_bytes = 2 * bpp * wl.params
+    stats_bytes = bpp * wl.params
+    proj_gbs = proj_bytes / (p_avg * 1e-3) / 1e9
+    stats_gbs = stats_bytes / (s_avg * 1e-3) / 1e9
+    tr_p, tr_s = recorded_traffic("gac_project_kernel"), recorded_traffic("gac_stats_kernel")
+    key = "bf16" if wl.g_dtype == torch.bfloat16 else "f32"
+    return {
+        "ms_per_step": step_ms, "stats_ms": s_avg, "project_ms": p_avg,
+        "best_ms_per_step": min(a + b for a, b in zip(s_ms, p_ms)),
+        "hbm_gbs": (proj_bytes + stats_bytes) / (step_ms * 1e-3) / 1e9,
+        "roofline": {"bound": "hbm", "kernel": "gac_project_kernel", "achieved": proj_gbs,
+                     "peak": peak, "unit": "GB/s", "frac": proj_gbs / peak,
+                     "peak_kind": f"of {peak_kind}", "frac_of_nominal_8TBs": proj_gbs / NOMINAL_HBM_GBS,
+                     "algorithmic_bytes_per_launch": proj_bytes,
+                     "traffic": (tr_p[key] * wl.params if tr_p and key in tr_p else None)},
+        "roofline_stats": {"bound": "hbm", "kernel": "gac_stats_kernel", "achieved": stats_gbs,
+                           "peak": peak, "unit": "GB/s", "frac": stats_gbs / peak,
+                           "peak_kind": f"of {peak_kind}",
+                           "algorithmic_bytes_per_launch": stats_bytes,
+                           "traffic": (tr_s[key] * wl.params if tr_s and key in tr_s else None)},
+    }
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="cfg3_7b_bf16", choices=sorted(synth.WORKLOADS))
+    ap.add_argument("--also", default="cfg5_14b_f32",
+                    help="second workload reported under 'also' (1 GPU only); 'none' to skip")
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.warmup < 3:
+        args.warmup = 3
+
+    if args.impl == "reference":
+        return run_reference(args)
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the GAC path has no CPU fallback")
+    from paper_2603_01501_b200 import binding as gb
+    gb.load_library()
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local_rank)
+    device = torch.device("cuda", local_rank)
+    if world > 1:
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        torch.distributed.init_process_group("nccl", device_id=device)
+    peak, peak_kind = measured_hbm_peak()
+
+    wl = Workload(args.workload, device, world)
+    sampler = ClockSampler(nvml_index(local_rank))
+    wall0 = time.perf_counter()
+    s_ms, p_ms = time_steps(wl, args.steps, args.warmup, sampler)
+    wall = time.perf_counter() - wall0
+    total_ms = sum(s_ms) + sum(p_ms)
+    if world > 1:
+        t = torch.tensor([total_ms], dtype=torch.float64, device=device)
+        torch.distributed.all_reduce(t, op=torch.distributed.ReduceOp.MAX)
+        total_ms = float(t.item())
+    res = check_regime(wl)
+    summ = summarize(wl, s_ms, p_ms, peak, peak_kind)
+    ms_per_step = total_ms / args.steps
+    info = gb.gac_get_info(wl.ctx)
+    line = {"metric": METRIC, "value": wl.params * world / (ms_per_step * 1e-3), "unit": UNIT,
+            "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_per_step,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32",
+            "data": "synthetic", "config": workload_config(args.workload, wl),
+            "hbm_gbs": summ["hbm_gbs"] , "frac_of_nominal_8TBs": summ["hbm_gbs"] / NOMINAL_HBM_GBS,
+            "stats_ms": summ["stats_ms"], "project_ms": summ["project_ms"],
+            "best_ms_per_step": summ["best_ms_per_step"],
+            "regime_check": {"cos": res.cos, "regime": gb.REGIME_NAMES[res.regime], "alpha": res.alpha},
+            "launch": {"grid": info.grid, "threads": info.threads, "chunk_elems": info.chunk_elems,
+                       "chunks": info.n_chunks},
+            "gpu_launches": (2 if world == 1 else 3) * args.steps,
+            "clocks": sampler.summary(), "roofline": summ["roofline"],
+            "roofline_stats": summ["roofline_stats"], "wall_s_timed_loop": wall}
+    if world > 1:
+        line["config"]["parallelism"] = (f"dp{world}: every rank holds one list as its gradient shard; "
+                                         "one NCCL all-reduce of 3 doubles per step")
+
+    if not args.no_e2e:
+        try:
+            line["e2e"] = time_e2e(wl, min(args.steps, 5), 1)
+            if world > 1:
+                t = torch.tensor([line["e2e"]["ms_per_step"]], dtype=torch.float64, device=device)
+                torch.distributed.all_reduce(t, op=torch.distributed.ReduceOp.MAX)
+                line["e2e"]["ms_per_step"] = float(t.item())
+                line["e2e"]["value"] = wl.params * world / (float(t.item()) * 1e-3)
+        except Exception as exc:  # host memory too small for the pinned copy, ...
+            line["e2e"] = {"value": None, "unit": UNIT, "error": repr(exc)[:200]}
+    wl.close()
+
+    if world == 1 and args.also != "none" and args.also != args.workload:
+        free, _ = torch.cuda.mem_get_info()
+        dims_key, g_dtype, _, _ = synth.WORKLOADS[args.also]
+        need = synth.list_numel(synth.decoder_tensor_list(synth.DIMS[dims_key])) * \
+            (bytes_per_param(g_dtype)) + (4 << 30)
+        if free > need:
+            wl2 = Workload(args.also, device, 1)
+            s2, p2 = time_steps(wl2, min(args.steps, 10), 3)
+            r2 = check_regime(wl2)
+            also = summarize(wl2, s2, p2, peak, peak_kind)
+            also.update({"workload": workload_config(args.also, wl2)["workload"],
+                         "params": wl2.params, "steps": min(args.steps, 10),
+                         "value": wl2.params / (also["ms_per_step"] * 1e-3), "unit": UNIT,
+                         "regime_check": {"cos": r2.cos, "regime": gb.REGIME_NAMES[r2.regime]}})
+            line["also"] = also
+            wl2.close()
+        else:
+            line["also"] = {"skipped": f"needs {need} bytes of device memory, {free} free"}
+
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        probe = time_oracle(args.workload, 8_000_000, 1, 0)
+        target = int(min(1_500_000_000, max(8_000_000, probe["value"] * 6.0)))
+        cb = time_oracle(args.workload, target, 2, 1)
+        line["cpu_baseline"] = {k: cb[k] for k in ("value", "unit", "cores", "kind", "sample")}
+
+    if world > 1:
+        torch.distributed.barrier()
+        torch.distributed.destroy_process_group()
+    if rank == 0:
+        print(json.dumps(line))
+    return 0
+
+
+if __name__ == "__main__":
+    sys.exit(main())

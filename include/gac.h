@@ -1,0 +1,201 @@
+/*
+ * gac.h -- C ABI of the B200 (sm_100a) library for the per-step hot path of
+ * Gradient Alignment Control (GAC).
+ *
+ * Notation follows the paper: g is the aggregated gradient of the current
+ * update step t (a list of per-parameter tensors, treated as one flattened
+ * concatenation, App. A.1), d is the stored snapshot of the previous step's
+ * gradient (App. A.2 "Memory footprint"), c_t their cosine (Eq. 1).
+ *
+ * Conventions for every entry point
+ *   - returns a gac_status; never throws, aborts or traps; on failure
+ *     gac_last_error() holds a message;
+ *   - "device pointer" = address in the memory of the CUDA device the context
+ *     was created for; "host pointer" = ordinary process memory;
+ *   - g and d buffers belong to the CALLER; the library reads/writes them only
+ *     inside gac_stats* / gac_project, on the stream given to that call;
+ *   - the context owns its chunk table, per-CTA partial sums, decision record
+ *     and a pinned host mirror of that record, and releases exactly those in
+ *     gac_free();
+ *   - one context serves one stream at a time and is not thread-safe.
+ */
+#ifndef GAC_H_
+#define GAC_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct gac_ctx gac_ctx;   /* opaque, library-owned */
+
+typedef enum {
+    GAC_OK = 0,
+    GAC_ERR_INVALID_ARG = 1,   /* null pointer, zero-length tensor, bad thresholds, ...      */
+    GAC_ERR_DTYPE = 2,         /* unsupported (g, d) element-type pair                       */
+    GAC_ERR_CUDA = 3,          /* a CUDA runtime call failed; message has the CUDA error     */
+    GAC_ERR_STATE = 4,         /* calls out of order (project without stats, step going back)*/
+    GAC_ERR_NONFINITE = 5,     /* NaN/Inf met in g or d; the step is reported as a violation  */
+    GAC_ERR_TIMEOUT = 6        /* reserved: no entry point of this library waits on the device */
+} gac_status;
+
+typedef enum { GAC_F32 = 0, GAC_BF16 = 1 } gac_dtype;
+
+/* The three regimes of Sec. 4.2 / Algorithm 1. */
+typedef enum { GAC_REGIME_SAFE = 0, GAC_REGIME_PROJECT = 1, GAC_REGIME_VIOLATION = 2 } gac_regime;
+
+typedef enum { GAC_MODE_ADAPTIVE = 0, GAC_MODE_FIXED = 1 } gac_mode;
+typedef enum { GAC_STATE_RAW = 0, GAC_STATE_PROJECTED = 1, GAC_STATE_HOLD = 2 } gac_state_mode;
+
+/* One parameter tensor: its gradient and its slot of the stored direction.
+ * Both are device pointers to `numel` contiguous elements, caller-owned.
+ * Any alignment is accepted; element-aligned is required, 16-byte aligned
+ * bases take the vectorised path. */
+typedef struct {
+    void *g;
+    void *d;
+    uint64_t numel;
+} gac_tensor;
+
+/* Hyper-parameters.  Defaults of the paper: c_low 0.05, c_high 0.3 (App. C.3),
+ * eps 1e-8 (App. A.1), beta 1 (App. A.2), adaptive mode, raw state. */
+typedef struct {
+    double c_low, c_high;      /* Algorithm 1 inputs; ADAPTIVE mode needs 0 < c_low < c_high.
+                                  c_high > 1 is legal and disables the skip branch.            */
+    double eps;                /* added to sqrt(<g,g><d,d>) in the cosine (App. A.1); >= 0     */
+    double beta;               /* gain of the orthogonal component (Eq. 3); finite             */
+    int32_t mode;              /* gac_mode: ADAPTIVE = Eq. 5 with the three regimes;
+                                  FIXED = Eq. 3 with (alpha_fixed, beta) on every step         */
+    int32_t state_mode;        /* gac_state_mode: RAW d' = g (the paper's rule);
+                                  PROJECTED d' = g'; HOLD d' = d                                */
+    double alpha_fixed;        /* gain of the parallel component in FIXED mode; 0 = remove it   */
+    int32_t zero_on_violation; /* 0: leave g alone, the caller skips its optimizer step
+                                  (Algorithm 1: theta_t = theta_{t-1}); 1: write g' = 0          */
+    int32_t reserved;          /* must be 0 */
+} gac_hparams;
+
+/* What one step decided.  Lives on the device between gac_stats and
+ * gac_project; copied to the host only when a host_out pointer is given. */
+typedef struct {
+    double dot, gg, dd;        /* <g,d>, <g,g>, <d,d> over the whole list (App. A.1)            */
+    double cos;                /* c_t = dot / (sqrt(gg*dd) + eps); 0 when gg or dd is 0          */
+    double alpha;              /* parallel gain used (Eq. 5: c_low/|c_t|); 1 when g is unchanged */
+    double coef64;             /* (alpha - beta) * dot / dd : multiplier of d in the rank-one
+                                  form g' = beta g + coef d (App. A.2)                          */
+    float coef;                /* coef64 rounded once to binary32: the value the kernel uses    */
+    int32_t regime;            /* gac_regime                                                    */
+    int32_t nonfinite;         /* 1 if a sum was NaN/Inf: regime = VIOLATION, g and d untouched  */
+    uint32_t staleness;        /* echoed metadata: the rule never reads it                      */
+    uint64_t step;             /* Algorithm 1's t for which this record holds                    */
+} gac_result;
+
+/* Fills *hp with the paper's defaults. */
+void gac_default_hparams(gac_hparams *hp);
+
+/*
+ * gac_init -- build a context for one list of parameter tensors.
+ * Presents the list as one logical flat vector (App. A.1: "flattened
+ * concatenation of all trainable parameter gradients") WITHOUT copying: the
+ * list is cut into fixed-size chunks, none spanning two tensors, and the chunk
+ * table is uploaded once.  Re-create the context if the tensors move.
+ *   out          host pointer, receives the context
+ *   list         host pointer to n entries (device pointers inside), copied
+ *   n            number of tensors, >= 1; every numel >= 1
+ *   g_dtype/d_dtype  supported pairs: (F32,F32), (BF16,F32)
+ *   hp           host pointer; copied
+ *   cuda_device  ordinal of the device that owns g and d
+ * Allocates device and pinned memory (not capturable in a CUDA graph).
+ * Errors: INVALID_ARG, DTYPE, CUDA.
+ */
+int gac_init(gac_ctx **out, const gac_tensor *list, uint32_t n, int g_dtype, int d_dtype,
+             const gac_hparams *hp, int cuda_device);
+
+/*
+ * gac_stats -- one fused pass over g and d: the three inner products of
+ * App. A.1, then the cosine with eps (App. A.1), the regime (Algorithm 1) and
+ * the gains (Eq. 5, or Eq. 3 in FIXED mode), all left in a device-resident
+ * decision record.  Sums are accumulated in binary64 in a fixed order: the
+ * same inputs give bit-identical results run to run.
+ *   step         Algorithm 1's t, counted from 1.  t = 1 means the stored
+ *                direction is g_0 = 0: d is NOT read (it may be uninitialised)
+ *                and the step is safe.  Must not go below the last step that
+ *                gac_project completed.
+ *   staleness    the lag tau of the behaviour policy; metadata only
+ *   cuda_stream  a cudaStream_t (or NULL for the default stream)
+ *   host_out     NULL: fully asynchronous, nothing leaves the device;
+ *                else the stream is synchronised and the record copied there
+ * Errors: INVALID_ARG, STATE, CUDA; NONFINITE only when host_out is given.
+ */
+int gac_stats(gac_ctx *ctx, uint64_t step, uint32_t staleness, void *cuda_stream,
+              gac_result *host_out);
+
+/*
+ * Sharded form of gac_stats for data-parallel gradient sharding (App. A.1,
+ * "Efficient computation under data parallelism"): each rank reduces its own
+ * shard, ONE all-reduce sums three numbers, every rank takes the same decision.
+ *   gac_stats_partial  writes this context's local (dot, gg, dd) to
+ *                      sums_out, a DEVICE pointer to 3 doubles owned by the
+ *                      caller, and takes no decision;
+ *   gac_decide         reads the GLOBAL (dot, gg, dd) from sums_in (device
+ *                      pointer to 3 doubles, e.g. after an all-reduce on the
+ *                      same stream) and fills the decision record.
+ * The collective between the two calls is the caller's.
+ */
+int gac_stats_partial(gac_ctx *ctx, uint64_t step, uint32_t staleness, void *cuda_stream,
+                      double *sums_out);
+int gac_decide(gac_ctx *ctx, void *cuda_stream, const double *sums_in, gac_result *host_out);
+
+/*
+ * gac_project -- one pass that reads g and d once and writes g' and d' in
+ * place, steered by the decision record on the device (no host round trip):
+ *   PROJECT regime   g'_i = beta g_i + coef d_i    (App. A.2 rank-one form;
+ *                    one fused multiply-add per element when beta = 1, result
+ *                    rounded to g's element type, nearest-even)
+ *   SAFE             g untouched (Algorithm 1: ordinary update)
+ *   VIOLATION        g untouched, or zeroed if zero_on_violation; the caller
+ *                    skips its optimizer step (Algorithm 1: theta_t = theta_{t-1})
+ *   every regime     d'_i = g_i, the raw gradient (state_mode RAW)
+ *   nonfinite        neither g nor d is written
+ * Must follow a gac_stats / gac_decide of the same step (else STATE).
+ *   coef_override    host pointer to one float, or NULL.  When given, it
+ *                    replaces the record's `coef` (used to compare outputs
+ *                    "given the same coefficient").
+ *   host_out         as in gac_stats
+ */
+int gac_project(gac_ctx *ctx, void *cuda_stream, const float *coef_override, gac_result *host_out);
+
+/* Releases what the context owns (never g or d).  NULL is accepted. */
+int gac_free(gac_ctx *ctx);
+
+/* Message of the last failure on this context; with ctx == NULL, of the last
+ * failed gac_init on the calling thread.  Never NULL. */
+const char *gac_last_error(const gac_ctx *ctx);
+
+/*
+ * Launch geometry (no counterpart in the paper; tuning only).  Values <= 0
+ * keep the default.  Must be called before the first gac_stats.
+ *   chunk_elems     elements per chunk (multiple of 1024)
+ *   ctas_per_sm     resident CTAs per SM the grid is sized for
+ * Changing them changes the summation order, hence the last bits of the sums.
+ */
+int gac_set_launch(gac_ctx *ctx, int chunk_elems, int ctas_per_sm);
+
+/* Facts about the context: total elements, chunks, grid size, kernel launches so far. */
+typedef struct {
+    uint64_t total_elems;
+    uint64_t n_chunks;
+    uint32_t n_tensors;
+    uint32_t grid;
+    uint32_t threads;
+    uint32_t chunk_elems;
+    uint64_t launches;
+    uint32_t misaligned_tensors;
+    uint32_t reserved;
+} gac_info;
+int gac_get_info(const gac_ctx *ctx, gac_info *out);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* GAC_H_ */

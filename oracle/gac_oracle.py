@@ -253,3 +253,42 @@ def round_to_bf16(x: np.ndarray) -> np.ndarray:
     out = np.empty(x.shape, dtype=np.uint16)
     lib().orc_round_to_bf16(x.ctypes.data, out.ctypes.data, x.size)
     return out
+
+
+class RunningStats:
+    """The same three sums, fed one tensor pair at a time so that a list larger
+    than host memory can be streamed through in list order."""
+
+    def __init__(self, first_step: bool = False, threads: int = 1):
+        self.first_step, self.threads = first_step, threads
+        self._tot = _Acc()
+        lib().orc_acc_init(ctypes.byref(self._tot))
+
+    def add(self, g, d) -> None:
+        L = lib()
+        gp, gdt, n = _ptr_dt_n(g)
+        dp, ddt, nd = _ptr_dt_n(d)
+        if n != nd:
+            raise ValueError("g and d differ in length")
+        fs = 1 if self.first_step else 0
+        jobs = [(gp + lo * _ELEM_BYTES[gdt], gdt, dp + lo * _ELEM_BYTES[ddt], ddt, hi - lo)
+                for lo, hi in _ranges(n, self.threads)]
+        if len(jobs) == 1:
+            j = jobs[0]
+            L.orc_stats_accumulate(ctypes.byref(self._tot), j[0], j[1], j[2], j[3], j[4], fs)
+            return
+
+        def run(j):
+            a = _Acc()
+            L.orc_acc_init(ctypes.byref(a))
+            L.orc_stats_accumulate(ctypes.byref(a), j[0], j[1], j[2], j[3], j[4], fs)
+            return a
+
+        with ThreadPoolExecutor(max_workers=self.threads) as ex:
+            for a in ex.map(run, jobs):
+                L.orc_acc_merge(ctypes.byref(self._tot), ctypes.byref(a))
+
+    def value(self):
+        out = (ctypes.c_double * 3)()
+        lib().orc_acc_value(ctypes.byref(self._tot), out)
+        return float(out[0]), float(out[1]), float(out[2])

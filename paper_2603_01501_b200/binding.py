@@ -1,0 +1,234 @@
+"""Thin ctypes binding of the C ABI in ``include/gac.h``: argument marshalling
+only.  Every step of the path runs in the CUDA library; if the library is
+missing this module raises -- there is no CPU fallback.
+
+PyTorch appears here only as the owner of device memory and streams.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from dataclasses import dataclass
+from typing import List, Optional, Sequence
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libgac_b200.so")
+
+GAC_OK, GAC_ERR_INVALID_ARG, GAC_ERR_DTYPE, GAC_ERR_CUDA, GAC_ERR_STATE, GAC_ERR_NONFINITE, \
+    GAC_ERR_TIMEOUT = range(7)
+GAC_F32, GAC_BF16 = 0, 1
+GAC_REGIME_SAFE, GAC_REGIME_PROJECT, GAC_REGIME_VIOLATION = 0, 1, 2
+GAC_MODE_ADAPTIVE, GAC_MODE_FIXED = 0, 1
+GAC_STATE_RAW, GAC_STATE_PROJECTED, GAC_STATE_HOLD = 0, 1, 2
+REGIME_NAMES = {0: "safe", 1: "project", 2: "violation"}
+
+
+class gac_tensor(ctypes.Structure):
+    _fields_ = [("g", ctypes.c_void_p), ("d", ctypes.c_void_p), ("numel", ctypes.c_uint64)]
+
+
+class gac_hparams(ctypes.Structure):
+    _fields_ = [("c_low", ctypes.c_double), ("c_high", ctypes.c_double), ("eps", ctypes.c_double),
+                ("beta", ctypes.c_double), ("mode", ctypes.c_int32), ("state_mode", ctypes.c_int32),
+                ("alpha_fixed", ctypes.c_double), ("zero_on_violation", ctypes.c_int32),
+                ("reserved", ctypes.c_int32)]
+
+
+class gac_result(ctypes.Structure):
+    _fields_ = [("dot", ctypes.c_double), ("gg", ctypes.c_double), ("dd", ctypes.c_double),
+                ("cos", ctypes.c_double), ("alpha", ctypes.c_double), ("coef64", ctypes.c_double),
+                ("coef", ctypes.c_float), ("regime", ctypes.c_int32), ("nonfinite", ctypes.c_int32),
+                ("staleness", ctypes.c_uint32), ("step", ctypes.c_uint64)]
+
+    def as_dict(self):
+        return {k: getattr(self, k) for k, _ in self._fields_}
+
+
+class gac_info(ctypes.Structure):
+    _fields_ = [("total_elems", ctypes.c_uint64), ("n_chunks", ctypes.c_uint64),
+                ("n_tensors", ctypes.c_uint32), ("grid", ctypes.c_uint32),
+                ("threads", ctypes.c_uint32), ("chunk_elems", ctypes.c_uint32),
+                ("launches", ctypes.c_uint64), ("misaligned_tensors", ctypes.c_uint32),
+                ("reserved", ctypes.c_uint32)]
+
+
+EXPORTS = ["gac_default_hparams", "gac_init", "gac_stats", "gac_stats_partial", "gac_decide",
+           "gac_project", "gac_free", "gac_last_error", "gac_set_launch", "gac_get_info"]
+
+_lib = None
+
+
+class GacError(RuntimeError):
+    def __init__(self, status: int, message: str):
+        super().__init__(f"gac status {status}: {message}")
+        self.status = status
+
+
+def load_library() -> ctypes.CDLL:
+    """Loads the in-tree CUDA library; raises if it was not built."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise ImportError(f"{LIB_PATH} is missing: build it with "
+                          "`python -m paper_2603_01501_b200.build` (needs nvcc); "
+                          "this package has no CPU fallback")
+    L = ctypes.CDLL(LIB_PATH)
+    vp, u32, u64, i32 = ctypes.c_void_p, ctypes.c_uint32, ctypes.c_uint64, ctypes.c_int
+    L.gac_default_hparams.argtypes = [ctypes.POINTER(gac_hparams)]
+    L.gac_default_hparams.restype = None
+    L.gac_init.argtypes = [ctypes.POINTER(vp), ctypes.POINTER(gac_tensor), u32, i32, i32,
+                           ctypes.POINTER(gac_hparams), i32]
+    L.gac_stats.argtypes = [vp, u64, u32, vp, ctypes.POINTER(gac_result)]
+    L.gac_stats_partial.argtypes = [vp, u64, u32, vp, vp]
+    L.gac_decide.argtypes = [vp, vp, vp, ctypes.POINTER(gac_result)]
+    L.gac_project.argtypes = [vp, vp, ctypes.POINTER(ctypes.c_float), ctypes.POINTER(gac_result)]
+    L.gac_free.argtypes = [vp]
+    L.gac_last_error.argtypes = [vp]
+    L.gac_last_error.restype = ctypes.c_char_p
+    L.gac_set_launch.argtypes = [vp, i32, i32]
+    L.gac_get_info.argtypes = [vp, ctypes.POINTER(gac_info)]
+    for name in ("gac_init", "gac_stats", "gac_stats_partial", "gac_decide", "gac_project",
+                 "gac_free", "gac_set_launch", "gac_get_info"):
+        getattr(L, name).restype = i32
+    _lib = L
+    return L
+
+
+@dataclass
+class HParams:
+    """Algorithm 1 inputs (c_low, c_high), the cosine's eps (App. A.1) and the
+    gains of Eq. 3 / Eq. 5; defaults are the paper's."""
+    c_low: float = 0.05
+    c_high: float = 0.3
+    eps: float = 1e-8
+    beta: float = 1.0
+    mode: int = GAC_MODE_ADAPTIVE
+    alpha_fixed: float = 0.0
+    state_mode: int = GAC_STATE_RAW
+    zero_on_violation: int = 0
+
+    def c(self) -> gac_hparams:
+        return gac_hparams(self.c_low, self.c_high, self.eps, self.beta, self.mode,
+                           self.state_mode, self.alpha_fixed, self.zero_on_violation, 0)
+
+
+_DT = {torch.float32: GAC_F32, torch.bfloat16: GAC_BF16}
+
+
+def _stream_ptr(stream) -> int:
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    return stream.cuda_stream if hasattr(stream, "cuda_stream") else int(stream)
+
+
+class GacContext:
+    """Owner of one ``gac_ctx``.  Keeps references to the tensors so that the
+    device pointers in the chunk table stay valid."""
+
+    def __init__(self, handle: int, g_list, d_list):
+        self.handle = ctypes.c_void_p(handle)
+        self._keep = (list(g_list), list(d_list))
+
+    def _check(self, rc: int, allow_nonfinite: bool = False):
+        if rc != GAC_OK and not (allow_nonfinite and rc == GAC_ERR_NONFINITE):
+            raise GacError(rc, load_library().gac_last_error(self.handle).decode())
+
+    def __del__(self):
+        try:
+            gac_free(self)
+        except Exception:
+            pass
+
+
+def gac_init(g_list: Sequence[torch.Tensor], d_list: Sequence[torch.Tensor],
+             hp: Optional[HParams] = None, device: Optional[int] = None) -> GacContext:
+    """gac_init of the C ABI on lists of CUDA tensors (g_i, d_i)."""
+    L = load_library()
+    hp = hp or HParams()
+    if len(g_list) != len(d_list):
+        raise ValueError("g and d lists differ in length")
+    n = len(g_list)
+    arr = (gac_tensor * max(n, 1))()
+    g_dt = d_dt = None
+    for i, (g, d) in enumerate(zip(g_list, d_list)):
+        if not (g.is_cuda and d.is_cuda and g.is_contiguous() and d.is_contiguous()):
+            raise ValueError("tensors must be contiguous CUDA tensors")
+        if g.numel() != d.numel():
+            raise ValueError(f"tensor {i}: g and d differ in numel")
+        if g.dtype not in _DT or d.dtype not in _DT:
+            raise GacError(GAC_ERR_DTYPE, f"unsupported dtype {g.dtype}/{d.dtype}")
+        if g_dt is None:
+            g_dt, d_dt = g.dtype, d.dtype
+        elif (g.dtype, d.dtype) != (g_dt, d_dt):
+            raise GacError(GAC_ERR_DTYPE, "all tensors of a list must share one (g,d) dtype pair")
+        arr[i] = gac_tensor(g.data_ptr(), d.data_ptr(), g.numel())
+    if device is None:
+        device = g_list[0].device.index if n else torch.cuda.current_device()
+    out = ctypes.c_void_p()
+    chp = hp.c()
+    rc = L.gac_init(ctypes.byref(out), arr, n, _DT.get(g_dt, 0), _DT.get(d_dt, 0),
+                    ctypes.byref(chp), device)
+    if rc != GAC_OK:
+        raise GacError(rc, L.gac_last_error(None).decode())
+    return GacContext(out.value, g_list, d_list)
+
+
+def gac_stats(ctx: GacContext, step: int, staleness: int = 0, stream=None,
+              fetch: bool = True) -> Optional[gac_result]:
+    """gac_stats; with fetch=False nothing leaves the device and None is returned."""
+    L = load_library()
+    res = gac_result() if fetch else None
+    rc = L.gac_stats(ctx.handle, step, staleness, _stream_ptr(stream),
+                     ctypes.byref(res) if fetch else None)
+    ctx._check(rc, allow_nonfinite=True)
+    return res
+
+
+def gac_stats_partial(ctx: GacContext, step: int, sums_out: torch.Tensor, staleness: int = 0,
+                      stream=None) -> None:
+    if not (sums_out.is_cuda and sums_out.dtype == torch.float64 and sums_out.numel() >= 3):
+        raise ValueError("sums_out must be a CUDA float64 tensor of 3 elements")
+    ctx._check(load_library().gac_stats_partial(ctx.handle, step, staleness, _stream_ptr(stream),
+                                                sums_out.data_ptr()))
+
+
+def gac_decide(ctx: GacContext, sums_in: torch.Tensor, stream=None,
+               fetch: bool = True) -> Optional[gac_result]:
+    if not (sums_in.is_cuda and sums_in.dtype == torch.float64 and sums_in.numel() >= 3):
+        raise ValueError("sums_in must be a CUDA float64 tensor of 3 elements")
+    res = gac_result() if fetch else None
+    rc = load_library().gac_decide(ctx.handle, _stream_ptr(stream), sums_in.data_ptr(),
+                                   ctypes.byref(res) if fetch else None)
+    ctx._check(rc, allow_nonfinite=True)
+    return res
+
+
+def gac_project(ctx: GacContext, stream=None, coef_override: Optional[float] = None,
+                fetch: bool = False) -> Optional[gac_result]:
+    L = load_library()
+    res = gac_result() if fetch else None
+    k = ctypes.c_float(coef_override) if coef_override is not None else None
+    rc = L.gac_project(ctx.handle, _stream_ptr(stream),
+                       ctypes.byref(k) if k is not None else None,
+                       ctypes.byref(res) if fetch else None)
+    ctx._check(rc, allow_nonfinite=True)
+    return res
+
+
+def gac_free(ctx: GacContext) -> None:
+    if ctx.handle:
+        load_library().gac_free(ctx.handle)
+        ctx.handle = ctypes.c_void_p(None)
+
+
+def gac_set_launch(ctx: GacContext, chunk_elems: int = 0, ctas_per_sm: int = 0) -> None:
+    ctx._check(load_library().gac_set_launch(ctx.handle, chunk_elems, ctas_per_sm))
+
+
+def gac_get_info(ctx: GacContext) -> gac_info:
+    info = gac_info()
+    ctx._check(load_library().gac_get_info(ctx.handle, ctypes.byref(info)))
+    return info

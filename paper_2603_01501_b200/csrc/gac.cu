@@ -1,0 +1,821 @@
+// CUDA implementation (sm_100a) of the GAC per-step hot path behind the C ABI in
+// include/gac.h.
+//
+//   chunk table      the list of parameter tensors is cut into fixed-size
+//                    chunks, none spanning two tensors; one launch walks them
+//                    all (App. A.1: the gradient is the flattened
+//                    concatenation of all parameter gradients -- presented
+//                    here without the flatten copy)
+//   gac_stats_kernel fused <g,d>, <g,g>, <d,d> (App. A.1) with binary64
+//                    accumulation, per-CTA partials, and a fixed-order second
+//                    stage run by the last CTA to finish, which also takes the
+//                    decision of Algorithm 1 / Eq. 5
+//   gac_project_kernel  g' = beta g + coef d in place and d' = g (App. A.2)
+//
+// The work is bound by HBM bandwidth: 3 FMAs per 8 bytes read in the first
+// pass, 1 FMA per 16 bytes moved in the second.  There is no dense contraction
+// here, hence no tensor-core path.
+#include <cuda_runtime.h>
+#include <math.h>
+#include <stdint.h>
+#include <stdio.h>
+#include <string.h>
+
+#include <algorithm>
+#include <new>
+#include <vector>
+
+#include "gac.h"
+
+namespace {
+
+constexpr int kThreads = 256;        // threads per CTA in both kernels
+constexpr int kUnroll = 4;           // 4-element vectors in flight per thread and operand
+constexpr int kDefaultChunk = 16384; // elements per chunk
+constexpr int kMaxCtasPerSm = 8;
+
+constexpr uint32_t kChunkAligned = 1u;  // both bases 16-byte aligned: vector path
+
+struct __align__(16) Chunk {
+    uint64_t g;      // device address of the chunk's first g element
+    uint64_t d;      // device address of the chunk's first d element
+    uint32_t n;      // elements in the chunk (<= chunk_elems)
+    uint32_t flags;
+    uint64_t pad;
+};
+static_assert(sizeof(Chunk) == 32, "chunk descriptors are read as two 16-byte words");
+
+// Hyper-parameters as the kernels see them.
+struct DevHP {
+    double c_low, c_high, eps, beta, alpha_fixed;
+    int mode, state_mode, zero_on_violation, first_step;
+    unsigned long long step;
+    unsigned staleness;
+    int decide;      // 0: only publish the three sums (sharded form)
+};
+
+struct F4 {
+    float x, y, z, w;
+};
+
+// ---------------------------------------------------------------- element I/O
+
+template <typename GT>
+struct Elem;
+
+template <>
+struct Elem<float> {
+    static __device__ __forceinline__ F4 load4(const void *base, uint32_t v) {
+        float4 t = reinterpret_cast<const float4 *>(base)[v];
+        return F4{t.x, t.y, t.z, t.w};
+    }
+    static __device__ __forceinline__ void store4(void *base, uint32_t v, F4 a) {
+        reinterpret_cast<float4 *>(base)[v] = make_float4(a.x, a.y, a.z, a.w);
+    }
+    static __device__ __forceinline__ float load1(const void *base, uint32_t i) {
+        return reinterpret_cast<const float *>(base)[i];
+    }
+    static __device__ __forceinline__ void store1(void *base, uint32_t i, float a) {
+        reinterpret_cast<float *>(base)[i] = a;
+    }
+};
+
+// bfloat16 = the upper 16 bits of a binary32 pattern.
+struct bf16_t {
+    uint16_t bits;
+};
+
+__device__ __forceinline__ uint32_t pack_bf16x2_rn(float lo, float hi) {
+    uint32_t r;
+    asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
+    return r;
+}
+
+template <>
+struct Elem<bf16_t> {
+    static __device__ __forceinline__ F4 load4(const void *base, uint32_t v) {
+        uint2 t = reinterpret_cast<const uint2 *>(base)[v];
+        return F4{__uint_as_float(t.x << 16), __uint_as_float(t.x & 0xFFFF0000u),
+                  __uint_as_float(t.y << 16), __uint_as_float(t.y & 0xFFFF0000u)};
+    }
+    static __device__ __forceinline__ void store4(void *base, uint32_t v, F4 a) {
+        reinterpret_cast<uint2 *>(base)[v] =
+            make_uint2(pack_bf16x2_rn(a.x, a.y), pack_bf16x2_rn(a.z, a.w));
+    }
+    static __device__ __forceinline__ float load1(const void *base, uint32_t i) {
+        return __uint_as_float(uint32_t(reinterpret_cast<const uint16_t *>(base)[i]) << 16);
+    }
+    static __device__ __forceinline__ void store1(void *base, uint32_t i, float a) {
+        reinterpret_cast<uint16_t *>(base)[i] = uint16_t(pack_bf16x2_rn(a, 0.0f) & 0xFFFFu);
+    }
+};
+
+__device__ __forceinline__ Chunk load_chunk(const Chunk *table, uint32_t c) {
+    const uint4 *p = reinterpret_cast<const uint4 *>(table + c);
+    uint4 a = __ldg(p), b = __ldg(p + 1);
+    Chunk ch;
+    ch.g = (uint64_t(a.y) << 32) | a.x;
+    ch.d = (uint64_t(a.w) << 32) | a.z;
+    ch.n = b.x;
+    ch.flags = b.y;
+    ch.pad = 0;
+    return ch;
+}
+
+// ------------------------------------------------------- decision (O(1) work)
+
+// Cosine with eps outside the root (App. A.1), the inclusive branches of
+// Algorithm 1, alpha = c_low/|c| (Eq. 5) or the caller's gain (Eq. 3), and the
+// multiplier of d in the rank-one form of App. A.2.
+__device__ void take_decision(double dot, double gg, double dd, const DevHP &hp, gac_result *r) {
+    if (hp.first_step) {   // Algorithm 1: g_0 = 0
+        dot = 0.0;
+        dd = 0.0;
+    }
+    r->dot = dot;
+    r->gg = gg;
+    r->dd = dd;
+    r->alpha = 1.0;
+    r->coef64 = 0.0;
+    r->coef = 0.0f;
+    r->staleness = hp.staleness;
+    r->step = hp.step;
+    r->nonfinite = !(isfinite(dot) && isfinite(gg) && isfinite(dd));
+    if (r->nonfinite) {
+        r->cos = __longlong_as_double(0x7FF8000000000000LL);
+        r->regime = GAC_REGIME_VIOLATION;
+        return;
+    }
+    if (gg == 0.0 || dd == 0.0) {   // zero reference: u = 0, projector = identity
+        r->cos = 0.0;
+        r->regime = GAC_REGIME_SAFE;
+        return;
+    }
+    double c = __ddiv_rn(dot, __dadd_rn(__dsqrt_rn(__dmul_rn(gg, dd)), hp.eps));
+    double ac = fabs(c);
+    r->cos = c;
+    if (hp.mode == GAC_MODE_FIXED) {
+        r->regime = GAC_REGIME_PROJECT;
+        r->alpha = hp.alpha_fixed;
+    } else if (ac <= hp.c_low) {
+        r->regime = GAC_REGIME_SAFE;
+        return;
+    } else if (ac >= hp.c_high) {
+        r->regime = GAC_REGIME_VIOLATION;
+        return;
+    } else {
+        r->regime = GAC_REGIME_PROJECT;
+        r->alpha = __ddiv_rn(hp.c_low, ac);
+    }
+    double k = __ddiv_rn(__dmul_rn(__dadd_rn(r->alpha, -hp.beta), dot), dd);
+    r->coef64 = k;
+    r->coef = __double2float_rn(k);
+}
+
+// ------------------------------------------------------------- stats kernel
+
+__device__ __forceinline__ double warp_sum(double v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xFFFFFFFFu, v, o);
+    return v;
+}
+
+// Sums (a, b, c) over the CTA in a fixed order; the result is valid in thread 0.
+__device__ __forceinline__ void block_sum3(double &a, double &b, double &c, double (*sm)[3]) {
+    a = warp_sum(a);
+    b = warp_sum(b);
+    c = warp_sum(c);
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    if (lane == 0) {
+        sm[warp][0] = a;
+        sm[warp][1] = b;
+        sm[warp][2] = c;
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        a = sm[0][0];
+        b = sm[0][1];
+        c = sm[0][2];
+        for (int w = 1; w < kThreads / 32; ++w) {
+            a += sm[w][0];
+            b += sm[w][1];
+            c += sm[w][2];
+        }
+    }
+    __syncthreads();
+}
+
+template <typename GT, bool READ_D>
+__device__ __forceinline__ void stats_chunk(const Chunk &ch, double &a_dot, double &a_gg,
+                                            double &a_dd) {
+    const void *g = reinterpret_cast<const void *>(ch.g);
+    const void *d = reinterpret_cast<const void *>(ch.d);
+    const uint32_t tid = threadIdx.x;
+    if (ch.flags & kChunkAligned) {
+        const uint32_t nvec = ch.n >> 2;
+        for (uint32_t base = 0; base < nvec; base += kThreads * kUnroll) {
+            F4 gv[kUnroll], dv[kUnroll];
+#pragma unroll
+            for (int u = 0; u < kUnroll; ++u) {
+                const uint32_t v = base + u * kThreads + tid;
+                if (v < nvec) {
+                    gv[u] = Elem<GT>::load4(g, v);
+                    if (READ_D) dv[u] = Elem<float>::load4(d, v);
+                } else {
+                    gv[u] = F4{0.f, 0.f, 0.f, 0.f};
+                    if (READ_D) dv[u] = F4{0.f, 0.f, 0.f, 0.f};
+                }
+            }
+#pragma unroll
+            for (int u = 0; u < kUnroll; ++u) {
+                const float ge[4] = {gv[u].x, gv[u].y, gv[u].z, gv[u].w};
+                const float de[4] = {dv[u].x, dv[u].y, dv[u].z, dv[u].w};
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    const double x = double(ge[e]);
+                    a_gg = fma(x, x, a_gg);
+                    if (READ_D) {
+                        const double y = double(de[e]);
+                        a_dot = fma(x, y, a_dot);
+                        a_dd = fma(y, y, a_dd);
+                    }
+                }
+            }
+        }
+        const uint32_t done = nvec << 2;
+        if (tid < ch.n - done) {   // ragged tail of a tensor: < 4 elements
+            const double x = double(Elem<GT>::load1(g, done + tid));
+            a_gg = fma(x, x, a_gg);
+            if (READ_D) {
+                const double y = double(Elem<float>::load1(d, done + tid));
+                a_dot = fma(x, y, a_dot);
+                a_dd = fma(y, y, a_dd);
+            }
+        }
+    } else {   // a base that is not 16-byte aligned: element-wise, still coalesced
+        for (uint32_t i = tid; i < ch.n; i += kThreads) {
+            const double x = double(Elem<GT>::load1(g, i));
+            a_gg = fma(x, x, a_gg);
+            if (READ_D) {
+                const double y = double(Elem<float>::load1(d, i));
+                a_dot = fma(x, y, a_dot);
+                a_dd = fma(y, y, a_dd);
+            }
+        }
+    }
+}
+
+// partials: gridDim.x x 3 doubles, each slot written once per launch.
+// ticket: zero on entry; the last CTA to arrive reduces the slots in index
+// order, publishes the result and puts the ticket back to zero.  No CTA waits.
+template <typename GT>
+__global__ void __launch_bounds__(kThreads)
+gac_stats_kernel(const Chunk *__restrict__ chunks, uint32_t n_chunks, double *partials,
+                 unsigned *ticket, gac_result *rec, double *sums_out, DevHP hp) {
+    __shared__ double sm[kThreads / 32][3];
+    __shared__ bool is_last;
+    double a_dot = 0.0, a_gg = 0.0, a_dd = 0.0;
+    if (hp.first_step) {
+        for (uint32_t c = blockIdx.x; c < n_chunks; c += gridDim.x)
+            stats_chunk<GT, false>(load_chunk(chunks, c), a_dot, a_gg, a_dd);
+    } else {
+        for (uint32_t c = blockIdx.x; c < n_chunks; c += gridDim.x)
+            stats_chunk<GT, true>(load_chunk(chunks, c), a_dot, a_gg, a_dd);
+    }
+    block_sum3(a_dot, a_gg, a_dd, sm);
+    if (threadIdx.x == 0) {
+        double *slot = partials + 3 * size_t(blockIdx.x);
+        slot[0] = a_dot;
+        slot[1] = a_gg;
+        slot[2] = a_dd;
+        __threadfence();
+        const unsigned t = atomicAdd(ticket, 1u);
+        is_last = (t == gridDim.x - 1);
+    }
+    __syncthreads();
+    if (!is_last) return;
+    __threadfence();
+    // second stage: thread t adds slots t, t+T, t+2T, ... in that order, then the
+    // same fixed tree as above
+    double s0 = 0.0, s1 = 0.0, s2 = 0.0;
+    for (uint32_t b = threadIdx.x; b < gridDim.x; b += kThreads) {
+        const double *slot = partials + 3 * size_t(b);
+        s0 += __ldcg(slot + 0);
+        s1 += __ldcg(slot + 1);
+        s2 += __ldcg(slot + 2);
+    }
+    block_sum3(s0, s1, s2, sm);
+    if (threadIdx.x == 0) {
+        *ticket = 0u;
+        if (sums_out) {
+            sums_out[0] = hp.first_step ? 0.0 : s0;
+            sums_out[1] = s1;
+            sums_out[2] = hp.first_step ? 0.0 : s2;
+        }
+        if (hp.decide) take_decision(s0, s1, s2, hp, rec);
+    }
+}
+
+__global__ void gac_decide_kernel(const double *sums_in, gac_result *rec, DevHP hp) {
+    if (threadIdx.x == 0 && blockIdx.x == 0)
+        take_decision(sums_in[0], sums_in[1], sums_in[2], hp, rec);
+}
+
+// ----------------------------------------------------------- project kernel
+
+enum GOp { G_KEEP = 0, G_FMA = 1, G_ZERO = 2 };
+enum DOp { D_KEEP = 0, D_RAW = 1, D_NEW = 2 };
+
+template <bool BETA1>
+__device__ __forceinline__ float rank_one(float g, float d, float k, double beta) {
+    if (BETA1) return fmaf(k, d, g);   // one rounding
+    // general beta: the sum of a rounded product and an exact product, in binary64
+    return __double2float_rn(__dadd_rn(__dmul_rn(beta, double(g)), __dmul_rn(double(k), double(d))));
+}
+
+template <typename GT, int GOP, int DOP, bool BETA1>
+__device__ __forceinline__ void project_chunk(const Chunk &ch, float k, double beta) {
+    void *g = reinterpret_cast<void *>(ch.g);
+    void *d = reinterpret_cast<void *>(ch.d);
+    const uint32_t tid = threadIdx.x;
+    constexpr bool kReadG = (GOP == G_FMA) || (DOP == D_RAW);
+    constexpr bool kReadD = (GOP == G_FMA);
+    if (ch.flags & kChunkAligned) {
+        const uint32_t nvec = ch.n >> 2;
+        for (uint32_t base = 0; base < nvec; base += kThreads * kUnroll) {
+            F4 gv[kUnroll], dv[kUnroll];
+#pragma unroll
+            for (int u = 0; u < kUnroll; ++u) {
+                const uint32_t v = base + u * kThreads + tid;
+                gv[u] = F4{0.f, 0.f, 0.f, 0.f};
+                dv[u] = F4{0.f, 0.f, 0.f, 0.f};
+                if (v < nvec) {
+                    if (kReadG) gv[u] = Elem<GT>::load4(g, v);
+                    if (kReadD) dv[u] = Elem<float>::load4(d, v);
+                }
+            }
+#pragma unroll
+            for (int u = 0; u < kUnroll; ++u) {
+                const uint32_t v = base + u * kThreads + tid;
+                if (v >= nvec) continue;
+                F4 out = gv[u];
+                if (GOP == G_FMA) {
+                    out.x = rank_one<BETA1>(gv[u].x, dv[u].x, k, beta);
+                    out.y = rank_one<BETA1>(gv[u].y, dv[u].y, k, beta);
+                    out.z = rank_one<BETA1>(gv[u].z, dv[u].z, k, beta);
+                    out.w = rank_one<BETA1>(gv[u].w, dv[u].w, k, beta);
+                }
+                if (GOP != G_KEEP) Elem<GT>::store4(g, v, out);
+                if (DOP == D_RAW) Elem<float>::store4(d, v, gv[u]);
+                if (DOP == D_NEW) {
+                    if (GOP == G_FMA) out = Elem<GT>::load4(g, v);   // the value as stored (rounded)
+                    Elem<float>::store4(d, v, out);
+                }
+            }
+        }
+        const uint32_t done = nvec << 2;
+        if (tid < ch.n - done) {
+            const uint32_t i = done + tid;
+            const float x = kReadG ? Elem<GT>::load1(g, i) : 0.f;
+            float out = x;
+            if (GOP == G_FMA) out = rank_one<BETA1>(x, Elem<float>::load1(d, i), k, beta);
+            if (GOP != G_KEEP) Elem<GT>::store1(g, i, out);
+            if (DOP == D_RAW) Elem<float>::store1(d, i, x);
+            if (DOP == D_NEW) {
+                if (GOP == G_FMA) out = Elem<GT>::load1(g, i);
+                Elem<float>::store1(d, i, out);
+            }
+        }
+    } else {
+        for (uint32_t i = tid; i < ch.n; i += kThreads) {
+            const float x = kReadG ? Elem<GT>::load1(g, i) : 0.f;
+            float out = x;
+            if (GOP == G_FMA) out = rank_one<BETA1>(x, Elem<float>::load1(d, i), k, beta);
+            if (GOP != G_KEEP) Elem<GT>::store1(g, i, out);
+            if (DOP == D_RAW) Elem<float>::store1(d, i, x);
+            if (DOP == D_NEW) {
+                if (GOP == G_FMA) out = Elem<GT>::load1(g, i);
+                Elem<float>::store1(d, i, out);
+            }
+        }
+    }
+}
+
+template <typename GT, int GOP, int DOP, bool BETA1>
+__device__ __forceinline__ void project_walk(const Chunk *chunks, uint32_t n_chunks, float k,
+                                             double beta) {
+    for (uint32_t c = blockIdx.x; c < n_chunks; c += gridDim.x)
+        project_chunk<GT, GOP, DOP, BETA1>(load_chunk(chunks, c), k, beta);
+}
+
+// The regime is read from the device-resident record, so no host round trip
+// separates the two passes.  Every CTA takes the same (uniform) branch.
+template <typename GT>
+__global__ void __launch_bounds__(kThreads)
+gac_project_kernel(const Chunk *__restrict__ chunks, uint32_t n_chunks, const gac_result *rec,
+                   float coef_override, int use_override, DevHP hp) {
+    if (rec->nonfinite) return;   // reading taken for NaN/Inf: touch nothing
+    const int regime = rec->regime;
+    const float k = use_override ? coef_override : rec->coef;
+    int gop = G_KEEP;
+    if (regime == GAC_REGIME_PROJECT) gop = G_FMA;
+    else if (regime == GAC_REGIME_VIOLATION && hp.zero_on_violation) gop = G_ZERO;
+    int dop = D_KEEP;
+    if (hp.state_mode == GAC_STATE_RAW) dop = D_RAW;
+    else if (hp.state_mode == GAC_STATE_PROJECTED) dop = (gop == G_KEEP) ? D_RAW : D_NEW;
+    const bool beta1 = (hp.beta == 1.0);
+
+    if (gop == G_FMA && dop == D_RAW && beta1) project_walk<GT, G_FMA, D_RAW, true>(chunks, n_chunks, k, 1.0);
+    else if (gop == G_KEEP && dop == D_RAW) project_walk<GT, G_KEEP, D_RAW, true>(chunks, n_chunks, k, 1.0);
+    else if (gop == G_KEEP && dop == D_KEEP) return;
+    else if (gop == G_FMA && dop == D_RAW) project_walk<GT, G_FMA, D_RAW, false>(chunks, n_chunks, k, hp.beta);
+    else if (gop == G_FMA && dop == D_NEW && beta1) project_walk<GT, G_FMA, D_NEW, true>(chunks, n_chunks, k, 1.0);
+    else if (gop == G_FMA && dop == D_NEW) project_walk<GT, G_FMA, D_NEW, false>(chunks, n_chunks, k, hp.beta);
+    else if (gop == G_FMA && dop == D_KEEP && beta1) project_walk<GT, G_FMA, D_KEEP, true>(chunks, n_chunks, k, 1.0);
+    else if (gop == G_FMA && dop == D_KEEP) project_walk<GT, G_FMA, D_KEEP, false>(chunks, n_chunks, k, hp.beta);
+    else if (gop == G_ZERO && dop == D_RAW) project_walk<GT, G_ZERO, D_RAW, true>(chunks, n_chunks, k, 1.0);
+    else if (gop == G_ZERO && dop == D_NEW) project_walk<GT, G_ZERO, D_NEW, true>(chunks, n_chunks, k, 1.0);
+    else if (gop == G_ZERO && dop == D_KEEP) project_walk<GT, G_ZERO, D_KEEP, true>(chunks, n_chunks, k, 1.0);
+}
+
+}  // namespace
+
+// ===================================================================== host
+
+struct gac_ctx {
+    int device = 0;
+    int g_dt = GAC_F32, d_dt = GAC_F32;
+    gac_hparams hp{};
+    std::vector<gac_tensor> list;
+    uint64_t total = 0;
+    uint32_t misaligned = 0;
+
+    Chunk *d_chunks = nullptr;
+    uint64_t n_chunks = 0;
+    double *d_partials = nullptr;
+    unsigned *d_ticket = nullptr;
+    gac_result *d_rec = nullptr;
+    gac_result *h_rec = nullptr;   // pinned
+
+    int sms = 0;
+    int chunk_elems = kDefaultChunk;
+    int ctas_per_sm = 0;           // 0 = what occupancy allows
+    int grid_stats = 0, grid_project = 0;
+
+    uint64_t last_projected_step = 0;
+    uint64_t pending_step = 0;
+    uint32_t pending_staleness = 0;
+    bool stats_pending = false;    // a partial reduction waits for gac_decide
+    bool decision_ready = false;   // a decision waits for gac_project
+    bool started = false;
+    uint64_t launches = 0;
+    char err[512] = {0};
+};
+
+namespace {
+
+thread_local char g_init_err[512] = "no error";
+
+int fail(gac_ctx *ctx, int code, const char *fmt, const char *a = "", long long b = 0) {
+    char *dst = ctx ? ctx->err : g_init_err;
+    snprintf(dst, 512, fmt, a, b);
+    return code;
+}
+
+struct DeviceGuard {
+    int prev = -1;
+    bool ok = true;
+    explicit DeviceGuard(int dev) {
+        if (cudaGetDevice(&prev) != cudaSuccess) prev = -1;
+        ok = (cudaSetDevice(dev) == cudaSuccess);
+    }
+    ~DeviceGuard() {
+        if (prev >= 0) cudaSetDevice(prev);
+    }
+};
+
+#define GAC_CUDA(ctx, call)                                                          \
+    do {                                                                             \
+        cudaError_t e_ = (call);                                                     \
+        if (e_ != cudaSuccess)                                                       \
+            return fail((ctx), GAC_ERR_CUDA, "%s (CUDA error %lld): " #call,        \
+                        cudaGetErrorString(e_), (long long)e_);                      \
+    } while (0)
+
+size_t elem_size(int dt) { return dt == GAC_BF16 ? 2 : 4; }
+
+void release_device(gac_ctx *c) {
+    if (c->d_chunks) cudaFree(c->d_chunks);
+    if (c->d_partials) cudaFree(c->d_partials);
+    if (c->d_ticket) cudaFree(c->d_ticket);
+    if (c->d_rec) cudaFree(c->d_rec);
+    if (c->h_rec) cudaFreeHost(c->h_rec);
+    c->d_chunks = nullptr;
+    c->d_partials = nullptr;
+    c->d_ticket = nullptr;
+    c->d_rec = nullptr;
+    c->h_rec = nullptr;
+}
+
+template <typename K>
+int resident_ctas(K kernel) {
+    int n = 0;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, kernel, kThreads, 0) != cudaSuccess || n < 1)
+        n = 1;
+    return std::min(n, kMaxCtasPerSm);
+}
+
+// Cuts the list into chunks and uploads the table; sizes both grids.
+int build_table(gac_ctx *c) {
+    const uint64_t ce = uint64_t(c->chunk_elems);
+    uint64_t n_chunks = 0;
+    for (const gac_tensor &t : c->list) n_chunks += (t.numel + ce - 1) / ce;
+    if (n_chunks > 0xFFFFFFF0ull)
+        return fail(c, GAC_ERR_INVALID_ARG, "too many chunks (%s%lld); raise chunk_elems", "",
+                    (long long)n_chunks);
+    std::vector<Chunk> table;
+    table.reserve(n_chunks);
+    const size_t gs = elem_size(c->g_dt), ds = elem_size(c->d_dt);
+    c->misaligned = 0;
+    for (const gac_tensor &t : c->list) {
+        const uint64_t gb = reinterpret_cast<uint64_t>(t.g), db = reinterpret_cast<uint64_t>(t.d);
+        const bool aligned = (gb % 16 == 0) && (db % 16 == 0);
+        if (!aligned) ++c->misaligned;
+        for (uint64_t off = 0; off < t.numel; off += ce) {
+            Chunk ch;
+            ch.g = gb + off * gs;
+            ch.d = db + off * ds;
+            ch.n = uint32_t(std::min<uint64_t>(ce, t.numel - off));
+            ch.flags = aligned ? kChunkAligned : 0u;
+            ch.pad = 0;
+            table.push_back(ch);
+        }
+    }
+    if (c->d_chunks) {
+        cudaFree(c->d_chunks);
+        c->d_chunks = nullptr;
+    }
+    GAC_CUDA(c, cudaMalloc(&c->d_chunks, table.size() * sizeof(Chunk)));
+    GAC_CUDA(c, cudaMemcpy(c->d_chunks, table.data(), table.size() * sizeof(Chunk),
+                           cudaMemcpyHostToDevice));
+    c->n_chunks = table.size();
+
+    int occ_s = c->g_dt == GAC_BF16 ? resident_ctas(gac_stats_kernel<bf16_t>)
+                                    : resident_ctas(gac_stats_kernel<float>);
+    int occ_p = c->g_dt == GAC_BF16 ? resident_ctas(gac_project_kernel<bf16_t>)
+                                    : resident_ctas(gac_project_kernel<float>);
+    if (c->ctas_per_sm > 0) {
+        occ_s = std::min(occ_s, c->ctas_per_sm);
+        occ_p = std::min(occ_p, c->ctas_per_sm);
+    }
+    c->grid_stats = int(std::min<uint64_t>(uint64_t(c->sms) * occ_s, c->n_chunks));
+    c->grid_project = int(std::min<uint64_t>(uint64_t(c->sms) * occ_p, c->n_chunks));
+    return GAC_OK;
+}
+
+int check_hparams(const gac_hparams *hp) {
+    if (!(hp->eps >= 0.0) || !isfinite(hp->eps)) return fail(nullptr, GAC_ERR_INVALID_ARG, "eps must be finite and >= 0%s");
+    if (!isfinite(hp->beta)) return fail(nullptr, GAC_ERR_INVALID_ARG, "beta must be finite%s");
+    if (hp->mode == GAC_MODE_ADAPTIVE) {
+        if (!(hp->c_low > 0.0) || !(hp->c_low < hp->c_high) || !isfinite(hp->c_high))
+            return fail(nullptr, GAC_ERR_INVALID_ARG, "thresholds must satisfy 0 < c_low < c_high%s");
+    } else if (hp->mode == GAC_MODE_FIXED) {
+        if (!(hp->alpha_fixed >= 0.0) || !isfinite(hp->alpha_fixed))
+            return fail(nullptr, GAC_ERR_INVALID_ARG, "alpha_fixed must be finite and >= 0%s");
+    } else {
+        return fail(nullptr, GAC_ERR_INVALID_ARG, "unknown mode%s");
+    }
+    if (hp->state_mode < GAC_STATE_RAW || hp->state_mode > GAC_STATE_HOLD)
+        return fail(nullptr, GAC_ERR_INVALID_ARG, "unknown state_mode%s");
+    if (hp->zero_on_violation != 0 && hp->zero_on_violation != 1)
+        return fail(nullptr, GAC_ERR_INVALID_ARG, "zero_on_violation must be 0 or 1%s");
+    if (hp->reserved != 0) return fail(nullptr, GAC_ERR_INVALID_ARG, "reserved field must be 0%s");
+    return GAC_OK;
+}
+
+DevHP dev_hp(const gac_ctx *c, uint64_t step, uint32_t staleness, int decide) {
+    DevHP h;
+    h.c_low = c->hp.c_low;
+    h.c_high = c->hp.c_high;
+    h.eps = c->hp.eps;
+    h.beta = c->hp.beta;
+    h.alpha_fixed = c->hp.alpha_fixed;
+    h.mode = c->hp.mode;
+    h.state_mode = c->hp.state_mode;
+    h.zero_on_violation = c->hp.zero_on_violation;
+    h.first_step = (step == 1);
+    h.step = step;
+    h.staleness = staleness;
+    h.decide = decide;
+    return h;
+}
+
+int read_back(gac_ctx *c, cudaStream_t s, gac_result *host_out) {
+    GAC_CUDA(c, cudaMemcpyAsync(c->h_rec, c->d_rec, sizeof(gac_result), cudaMemcpyDeviceToHost, s));
+    GAC_CUDA(c, cudaStreamSynchronize(s));
+    *host_out = *c->h_rec;
+    if (host_out->nonfinite)
+        return fail(c, GAC_ERR_NONFINITE, "NaN or Inf met in the gradient or the stored direction%s");
+    return GAC_OK;
+}
+
+int launch_stats(gac_ctx *c, uint64_t step, uint32_t staleness, cudaStream_t s, double *sums_out,
+                 int decide) {
+    if (step == 0) return fail(c, GAC_ERR_INVALID_ARG, "step counts from 1 (Algorithm 1)%s");
+    if (c->started && step <= c->last_projected_step)
+        return fail(c, GAC_ERR_STATE, "step %s%lld was already projected", "", (long long)step);
+    const DevHP h = dev_hp(c, step, staleness, decide);
+    const uint32_t nc = uint32_t(c->n_chunks);
+    if (c->g_dt == GAC_BF16)
+        gac_stats_kernel<bf16_t><<<c->grid_stats, kThreads, 0, s>>>(c->d_chunks, nc, c->d_partials,
+                                                                    c->d_ticket, c->d_rec, sums_out, h);
+    else
+        gac_stats_kernel<float><<<c->grid_stats, kThreads, 0, s>>>(c->d_chunks, nc, c->d_partials,
+                                                                   c->d_ticket, c->d_rec, sums_out, h);
+    GAC_CUDA(c, cudaGetLastError());
+    ++c->launches;
+    c->pending_step = step;
+    return GAC_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+void gac_default_hparams(gac_hparams *hp) {
+    if (!hp) return;
+    memset(hp, 0, sizeof(*hp));
+    hp->c_low = 0.05;
+    hp->c_high = 0.3;
+    hp->eps = 1e-8;
+    hp->beta = 1.0;
+    hp->mode = GAC_MODE_ADAPTIVE;
+    hp->state_mode = GAC_STATE_RAW;
+}
+
+int gac_init(gac_ctx **out, const gac_tensor *list, uint32_t n, int g_dtype, int d_dtype,
+             const gac_hparams *hp, int cuda_device) {
+    if (!out) return fail(nullptr, GAC_ERR_INVALID_ARG, "out is NULL%s");
+    *out = nullptr;
+    if (!list || n == 0) return fail(nullptr, GAC_ERR_INVALID_ARG, "empty tensor list%s");
+    if (!hp) return fail(nullptr, GAC_ERR_INVALID_ARG, "hp is NULL%s");
+    if (!((g_dtype == GAC_F32 || g_dtype == GAC_BF16) && d_dtype == GAC_F32))
+        return fail(nullptr, GAC_ERR_DTYPE, "supported (g,d) element types: (f32,f32), (bf16,f32)%s");
+    if (int rc = check_hparams(hp)) return rc;
+    const size_t gs = elem_size(g_dtype), ds = elem_size(d_dtype);
+    for (uint32_t i = 0; i < n; ++i) {
+        if (!list[i].g || !list[i].d)
+            return fail(nullptr, GAC_ERR_INVALID_ARG, "tensor %s%lld has a NULL pointer", "", i);
+        if (list[i].numel == 0)
+            return fail(nullptr, GAC_ERR_INVALID_ARG, "tensor %s%lld has no elements", "", i);
+        if (list[i].numel > (1ull << 40))
+            return fail(nullptr, GAC_ERR_INVALID_ARG, "tensor %s%lld is larger than 2^40 elements", "", i);
+        const uint64_t gb = reinterpret_cast<uint64_t>(list[i].g), db = reinterpret_cast<uint64_t>(list[i].d);
+        if (gb % gs || db % ds)
+            return fail(nullptr, GAC_ERR_INVALID_ARG, "tensor %s%lld is not element-aligned", "", i);
+        // g is updated in place while d is read: the two ranges must not overlap
+        if (gb < db + list[i].numel * ds && db < gb + list[i].numel * gs)
+            return fail(nullptr, GAC_ERR_INVALID_ARG, "tensor %s%lld: g and d overlap", "", i);
+    }
+    int n_dev = 0;
+    if (cudaGetDeviceCount(&n_dev) != cudaSuccess || n_dev == 0)
+        return fail(nullptr, GAC_ERR_CUDA, "no CUDA device is available%s");
+    if (cuda_device < 0 || cuda_device >= n_dev)
+        return fail(nullptr, GAC_ERR_INVALID_ARG, "cuda_device %s%lld out of range", "", cuda_device);
+
+    gac_ctx *c = new (std::nothrow) gac_ctx;
+    if (!c) return fail(nullptr, GAC_ERR_INVALID_ARG, "out of host memory%s");
+    c->device = cuda_device;
+    c->g_dt = g_dtype;
+    c->d_dt = d_dtype;
+    c->hp = *hp;
+    c->list.assign(list, list + n);
+    for (uint32_t i = 0; i < n; ++i) c->total += list[i].numel;
+
+    DeviceGuard guard(cuda_device);
+    int rc = GAC_OK;
+    auto setup = [&]() -> int {
+        if (!guard.ok) return fail(c, GAC_ERR_CUDA, "cudaSetDevice failed%s");
+        GAC_CUDA(c, cudaDeviceGetAttribute(&c->sms, cudaDevAttrMultiProcessorCount, cuda_device));
+        // small inputs: shorter chunks so that every SM still gets work
+        while (c->chunk_elems > 4096 && c->total / uint64_t(c->chunk_elems) < uint64_t(4 * c->sms))
+            c->chunk_elems /= 2;
+        if (int r = build_table(c)) return r;
+        GAC_CUDA(c, cudaMalloc(&c->d_partials, size_t(c->sms) * kMaxCtasPerSm * 3 * sizeof(double)));
+        GAC_CUDA(c, cudaMalloc(&c->d_ticket, sizeof(unsigned)));
+        GAC_CUDA(c, cudaMemset(c->d_ticket, 0, sizeof(unsigned)));
+        GAC_CUDA(c, cudaMalloc(&c->d_rec, sizeof(gac_result)));
+        GAC_CUDA(c, cudaMemset(c->d_rec, 0, sizeof(gac_result)));
+        GAC_CUDA(c, cudaMallocHost(&c->h_rec, sizeof(gac_result)));
+        return GAC_OK;
+    };
+    rc = setup();
+    if (rc != GAC_OK) {
+        memcpy(g_init_err, c->err, sizeof(g_init_err));
+        release_device(c);
+        delete c;
+        return rc;
+    }
+    *out = c;
+    return GAC_OK;
+}
+
+int gac_set_launch(gac_ctx *ctx, int chunk_elems, int ctas_per_sm) {
+    if (!ctx) return fail(nullptr, GAC_ERR_INVALID_ARG, "ctx is NULL%s");
+    if (ctx->started) return fail(ctx, GAC_ERR_STATE, "launch geometry is fixed once a step has run%s");
+    if (chunk_elems > 0) {
+        if (chunk_elems % 1024) return fail(ctx, GAC_ERR_INVALID_ARG, "chunk_elems must be a multiple of 1024%s");
+        ctx->chunk_elems = chunk_elems;
+    }
+    if (ctas_per_sm > 0) ctx->ctas_per_sm = std::min(ctas_per_sm, kMaxCtasPerSm);
+    DeviceGuard guard(ctx->device);
+    return build_table(ctx);
+}
+
+int gac_stats(gac_ctx *ctx, uint64_t step, uint32_t staleness, void *cuda_stream, gac_result *host_out) {
+    if (!ctx) return fail(nullptr, GAC_ERR_INVALID_ARG, "ctx is NULL%s");
+    DeviceGuard guard(ctx->device);
+    cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+    if (int rc = launch_stats(ctx, step, staleness, s, nullptr, 1)) return rc;
+    ctx->started = true;
+    ctx->stats_pending = false;
+    ctx->decision_ready = true;
+    return host_out ? read_back(ctx, s, host_out) : GAC_OK;
+}
+
+int gac_stats_partial(gac_ctx *ctx, uint64_t step, uint32_t staleness, void *cuda_stream, double *sums_out) {
+    if (!ctx) return fail(nullptr, GAC_ERR_INVALID_ARG, "ctx is NULL%s");
+    if (!sums_out) return fail(ctx, GAC_ERR_INVALID_ARG, "sums_out is NULL%s");
+    DeviceGuard guard(ctx->device);
+    cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+    if (int rc = launch_stats(ctx, step, staleness, s, sums_out, 0)) return rc;
+    ctx->started = true;
+    ctx->stats_pending = true;
+    ctx->decision_ready = false;
+    ctx->pending_staleness = staleness;
+    return GAC_OK;
+}
+
+int gac_decide(gac_ctx *ctx, void *cuda_stream, const double *sums_in, gac_result *host_out) {
+    if (!ctx) return fail(nullptr, GAC_ERR_INVALID_ARG, "ctx is NULL%s");
+    if (!sums_in) return fail(ctx, GAC_ERR_INVALID_ARG, "sums_in is NULL%s");
+    if (!ctx->stats_pending) return fail(ctx, GAC_ERR_STATE, "gac_decide needs a gac_stats_partial first%s");
+    DeviceGuard guard(ctx->device);
+    cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+    const DevHP h = dev_hp(ctx, ctx->pending_step, ctx->pending_staleness, 1);
+    gac_decide_kernel<<<1, 32, 0, s>>>(sums_in, ctx->d_rec, h);
+    GAC_CUDA(ctx, cudaGetLastError());
+    ++ctx->launches;
+    ctx->stats_pending = false;
+    ctx->decision_ready = true;
+    return host_out ? read_back(ctx, s, host_out) : GAC_OK;
+}
+
+int gac_project(gac_ctx *ctx, void *cuda_stream, const float *coef_override, gac_result *host_out) {
+    if (!ctx) return fail(nullptr, GAC_ERR_INVALID_ARG, "ctx is NULL%s");
+    if (!ctx->decision_ready)
+        return fail(ctx, GAC_ERR_STATE, "gac_project needs the decision of gac_stats / gac_decide for this step%s");
+    DeviceGuard guard(ctx->device);
+    cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+    const DevHP h = dev_hp(ctx, ctx->pending_step, 0, 1);
+    const float k = coef_override ? *coef_override : 0.0f;
+    const int use = coef_override ? 1 : 0;
+    const uint32_t nc = uint32_t(ctx->n_chunks);
+    if (ctx->g_dt == GAC_BF16)
+        gac_project_kernel<bf16_t><<<ctx->grid_project, kThreads, 0, s>>>(ctx->d_chunks, nc, ctx->d_rec, k, use, h);
+    else
+        gac_project_kernel<float><<<ctx->grid_project, kThreads, 0, s>>>(ctx->d_chunks, nc, ctx->d_rec, k, use, h);
+    GAC_CUDA(ctx, cudaGetLastError());
+    ++ctx->launches;
+    ctx->decision_ready = false;
+    ctx->last_projected_step = ctx->pending_step;
+    return host_out ? read_back(ctx, s, host_out) : GAC_OK;
+}
+
+int gac_free(gac_ctx *ctx) {
+    if (!ctx) return GAC_OK;
+    {
+        DeviceGuard guard(ctx->device);
+        release_device(ctx);
+    }
+    delete ctx;
+    return GAC_OK;
+}
+
+const char *gac_last_error(const gac_ctx *ctx) { return ctx ? ctx->err : g_init_err; }
+
+int gac_get_info(const gac_ctx *ctx, gac_info *out) {
+    if (!ctx || !out) return GAC_ERR_INVALID_ARG;
+    out->total_elems = ctx->total;
+    out->n_chunks = ctx->n_chunks;
+    out->n_tensors = uint32_t(ctx->list.size());
+    out->grid = uint32_t(ctx->grid_stats);
+    out->threads = kThreads;
+    out->chunk_elems = uint32_t(ctx->chunk_elems);
+    out->launches = ctx->launches;
+    out->misaligned_tensors = ctx->misaligned;
+    out->reserved = 0;
+    return GAC_OK;
+}
+
+}  // extern "C"

@@ -193,3 +193,28 @@ class StalenessProcess:
         if len(self.window) > self.k:
             self.window.pop(0)
         return g
+
+
+def refresh_gradient_list(g_list: Sequence[torch.Tensor], d_list: Sequence[torch.Tensor],
+                          sigma: Sequence[float], rho: float, gen: torch.Generator,
+                          scratch: torch.Tensor) -> None:
+    """Overwrites every g_i with a fresh gradient whose expected cosine to the
+    current stored direction is rho: g_i = rho d_i + sqrt(1-rho^2) sigma_i w,
+    w ~ N(0,1) (one AR(1) step of the staleness process).  `scratch` is a
+    float32 work buffer at least as long as the largest tensor."""
+    c = math.sqrt(1.0 - rho * rho)
+    for g, d, s in zip(g_list, d_list, sigma):
+        w = scratch[: g.numel()]
+        w.normal_(generator=gen)
+        w.mul_(c * s).add_(d, alpha=rho)
+        g.copy_(w)
+
+
+WORKLOADS = {
+    # name: (dims key, g dtype, rho, config id)  -- the decoder-shaped lists of the benchmark
+    "cfg2_1.5b_f32": ("1.5b", torch.float32, 0.8, 2),
+    "cfg3_7b_bf16": ("7b", torch.bfloat16, 0.95, 3),
+    "cfg5_14b_f32": ("14b", torch.float32, 0.9, 5),
+    "small_f32": ("small", torch.float32, 0.9, 2),
+    "small_bf16": ("small", torch.bfloat16, 0.95, 3),
+}

@@ -1,0 +1,293 @@
+"""GPU parity: the CUDA library, called through its C ABI, against the CPU
+oracle on the same seeded inputs, element by element."""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import gac_oracle as orc
+from paper_2603_01501_b200 import binding as gb
+from paper_2603_01501_b200 import synth
+
+from gpu_util import (check_decision, check_outputs, check_sums, max_ulp, step_both, to_orc_hp)
+
+pytestmark = pytest.mark.gpu
+
+FORCE = dict(c_low=0.05, c_high=2.0)      # legal (c_high > 1): every |c| > c_low is projected
+
+
+def rand_pair(n, rho, seed, g_dtype=torch.float32, scale=1.0):
+    gen = torch.Generator().manual_seed(seed)
+    d = torch.randn(n, generator=gen) * scale
+    w = torch.randn(n, generator=gen) * scale
+    g = (rho * d + math.sqrt(max(0.0, 1 - rho * rho)) * w).to(g_dtype)
+    return g, d
+
+
+# ------------------------------------------------------------------ config 1
+
+@pytest.mark.parametrize("hp", [gb.HParams(), gb.HParams(**FORCE),
+                                gb.HParams(mode=gb.GAC_MODE_FIXED, alpha_fixed=0.0)],
+                         ids=["defaults", "forced_projection", "full_projection"])
+def test_flat_pair_2pow20(hp):
+    g, d = synth.flat_pair_with_cosine(1 << 20, 0.9, s=1.0, seed=0)
+    res, dec, gg, dg, gr, dr = step_both([g], [d], hp)
+    check_sums(res, dec)
+    check_decision(res, dec)
+    assert abs(res.cos - 0.9) < 1e-6
+    assert res.regime == (gb.GAC_REGIME_VIOLATION if hp.mode == 0 and hp.c_high < 0.9
+                          else gb.GAC_REGIME_PROJECT)
+    check_outputs(gg, dg, gr, dr)
+    if hp.mode == gb.GAC_MODE_FIXED:      # g' orthogonal to d after a full projection
+        d64 = d.double()
+        assert abs(float(torch.dot(gg[0].cpu().double(), d64))) <= 1e-6 * math.sqrt(res.gg * res.dd)
+
+
+# ------------------------------------------------- sizes, tails, several tiles
+
+SIZES = [1, 2, 3, 4, 5, 7, 255, 256, 1023, 1024, 1025, 4095, 4096, 4097, 16383, 16384, 16385,
+         5 * 16384 + 7, 1_000_003]
+
+
+@pytest.mark.parametrize("g_dtype", [torch.float32, torch.bfloat16], ids=["f32", "bf16"])
+@pytest.mark.parametrize("n", SIZES)
+def test_single_tensor_sizes(n, g_dtype):
+    g, d = rand_pair(n, 0.5, seed=n, g_dtype=g_dtype, scale=0.01)
+    res, dec, gg, dg, gr, dr = step_both([g], [d], gb.HParams(**FORCE))
+    check_sums(res, dec)
+    check_decision(res, dec)
+    check_outputs(gg, dg, gr, dr)
+
+
+@pytest.mark.parametrize("g_dtype", [torch.float32, torch.bfloat16], ids=["f32", "bf16"])
+@pytest.mark.parametrize("name,rho", [("mini", 0.2), ("small", 0.8)])
+def test_decoder_shaped_lists(name, rho, g_dtype):
+    shapes = synth.decoder_tensor_list(synth.DIMS[name])
+    g, d = synth.gradient_list(shapes, rho, config_id=2, g_dtype=g_dtype)
+    for hp in (gb.HParams(), gb.HParams(**FORCE)):
+        res, dec, gg, dg, gr, dr = step_both(g, d, hp)
+        check_sums(res, dec)
+        check_decision(res, dec)
+        check_outputs(gg, dg, gr, dr)
+        assert abs(res.cos - rho) < 0.02
+
+
+@pytest.mark.parametrize("launch", [(1024, 1), (4096, 2), (65536, 8)])
+def test_launch_geometry_does_not_change_results(launch):
+    shapes = synth.decoder_tensor_list(synth.DIMS["small"])
+    g, d = synth.gradient_list(shapes, 0.6, config_id=2)
+    res, dec, gg, dg, gr, dr = step_both(g, d, gb.HParams(**FORCE), launch=launch)
+    check_sums(res, dec, rel=1e-12)
+    check_decision(res, dec)
+    check_outputs(gg, dg, gr, dr)
+
+
+@pytest.mark.parametrize("g_dtype", [torch.float32, torch.bfloat16], ids=["f32", "bf16"])
+def test_misaligned_views_and_guard_regions(g_dtype):
+    """Tensors that start at odd element offsets inside larger buffers (views):
+    the element-wise path must give the same results, and nothing outside the
+    views may be touched."""
+    torch.manual_seed(5)
+    sizes = [1, 3, 1000, 16384, 40001]
+    offs = [1, 3, 5, 2, 7]
+    hp = gb.HParams(**FORCE)
+    g_cpu, d_cpu, g_buf, d_buf, g_view, d_view = [], [], [], [], [], []
+    for n, o in zip(sizes, offs):
+        g, d = rand_pair(n, 0.4, seed=n + 1, g_dtype=g_dtype)
+        g_cpu.append(g)
+        d_cpu.append(d)
+        gbuf = torch.full((n + 16,), 7.0, dtype=g_dtype, device="cuda")
+        dbuf = torch.full((n + 16,), -9.0, dtype=torch.float32, device="cuda")
+        gbuf[o:o + n] = g.cuda()
+        dbuf[o + 1:o + 1 + n] = d.cuda()
+        g_buf.append(gbuf)
+        d_buf.append(dbuf)
+        g_view.append(gbuf[o:o + n])
+        d_view.append(dbuf[o + 1:o + 1 + n])
+    ohp = to_orc_hp(hp)
+    g_ref, d_ref = [t.clone() for t in g_cpu], [t.clone() for t in d_cpu]
+    dec = orc.step(g_ref, d_ref, ohp)
+    ctx = gb.gac_init(g_view, d_view, hp)
+    assert gb.gac_get_info(ctx).misaligned_tensors == len(sizes)
+    res = gb.gac_stats(ctx, 2)
+    gb.gac_project(ctx, coef_override=dec.coef)
+    torch.cuda.synchronize()
+    check_sums(res, dec)
+    check_decision(res, dec)
+    check_outputs(g_view, d_view, g_ref, d_ref)
+    for n, o, gbuf, dbuf in zip(sizes, offs, g_buf, d_buf):
+        assert bool((gbuf[:o] == 7.0).all()) and bool((gbuf[o + n:] == 7.0).all())
+        assert bool((dbuf[:o + 1] == -9.0).all()) and bool((dbuf[o + 1 + n:] == -9.0).all())
+
+
+# ------------------------------------------------------- regimes and readings
+
+def test_three_regimes_and_raw_state_over_steps():
+    torch.manual_seed(1)
+    n = 70_001
+    hp = gb.HParams()           # paper defaults 0.05 / 0.3
+    d0 = torch.randn(n)
+    d_gpu = [torch.full((n,), float("nan"), device="cuda")]      # never read on step 1
+    g_gpu = [torch.empty(n, device="cuda")]
+    ctx = gb.gac_init(g_gpu, d_gpu, hp)
+    d_ref = [torch.full((n,), float("nan"))]
+    seen = []
+    prev = d0
+    for t, rho in enumerate([None, 0.0, 0.15, 0.8, 0.02, 0.2], start=1):
+        g = torch.randn(n) if rho is None else rho * prev + math.sqrt(1 - rho * rho) * torch.randn(n)
+        prev = g.clone()
+        g_gpu[0].copy_(g)
+        g_ref = [g.clone()]
+        dec = orc.step(g_ref, d_ref, to_orc_hp(hp), first_step=(t == 1))
+        res = gb.gac_stats(ctx, t, staleness=t % 3)
+        gb.gac_project(ctx, coef_override=dec.coef if dec.regime == orc.PROJECT else None)
+        assert res.step == t and res.staleness == t % 3
+        if t == 1:
+            assert (res.dot, res.dd, res.cos, res.regime) == (0.0, 0.0, 0.0, gb.GAC_REGIME_SAFE)
+        check_sums(res, dec)
+        check_decision(res, dec)
+        check_outputs(g_gpu, d_gpu, g_ref, d_ref)
+        assert torch.equal(d_gpu[0].cpu(), g)               # state = raw gradient, every regime
+        seen.append(res.regime)
+    assert set(seen) == {0, 1, 2}
+    gb.gac_free(ctx)
+
+
+@pytest.mark.parametrize("hp", [
+    gb.HParams(zero_on_violation=1),
+    gb.HParams(**FORCE, state_mode=gb.GAC_STATE_PROJECTED),
+    gb.HParams(**FORCE, state_mode=gb.GAC_STATE_HOLD),
+    gb.HParams(mode=gb.GAC_MODE_FIXED, alpha_fixed=0.25, beta=1.5),
+    gb.HParams(mode=gb.GAC_MODE_FIXED, alpha_fixed=2.0, beta=0.5, state_mode=gb.GAC_STATE_PROJECTED),
+    gb.HParams(zero_on_violation=1, state_mode=gb.GAC_STATE_PROJECTED),
+    gb.HParams(zero_on_violation=1, state_mode=gb.GAC_STATE_HOLD),
+    gb.HParams(state_mode=gb.GAC_STATE_HOLD),
+], ids=["zero_on_violation", "projected_state", "hold_state", "fixed_gains", "fixed_gains_projected",
+        "zero_projected", "zero_hold", "violation_hold"])
+@pytest.mark.parametrize("g_dtype", [torch.float32, torch.bfloat16], ids=["f32", "bf16"])
+def test_variants(hp, g_dtype):
+    g, d = rand_pair(50_003, 0.7, seed=3, g_dtype=g_dtype)
+    res, dec, gg, dg, gr, dr = step_both([g], [d], hp)
+    check_sums(res, dec)
+    check_decision(res, dec)
+    check_outputs(gg, dg, gr, dr)
+
+
+def test_degenerate_vectors():
+    n = 5000
+    g, d = rand_pair(n, 0.5, seed=9)
+    z = torch.zeros(n)
+    for gv, dv in [(g, z), (z, d), (z, z), (g, g.clone()), (g, -g)]:
+        for hp in (gb.HParams(), gb.HParams(eps=0.0)):
+            res, dec, gg, dg, gr, dr = step_both([gv.clone()], [dv.clone()], hp)
+            check_sums(res, dec)
+            check_decision(res, dec)
+            check_outputs(gg, dg, gr, dr)
+    res, *_ = step_both([g], [g.clone()], gb.HParams(eps=0.0))
+    assert abs(res.cos - 1.0) < 1e-12 and res.regime == gb.GAC_REGIME_VIOLATION
+
+
+def test_nonfinite_is_reported_and_nothing_is_written():
+    g, d = rand_pair(10_000, 0.5, seed=2)
+    g[1234] = float("inf")
+    g_gpu, d_gpu = [g.cuda()], [d.cuda()]
+    ctx = gb.gac_init(g_gpu, d_gpu, gb.HParams())
+    res = gb.gac_stats(ctx, 2)
+    gb.gac_project(ctx)
+    torch.cuda.synchronize()
+    assert res.nonfinite == 1 and res.regime == gb.GAC_REGIME_VIOLATION
+    assert torch.equal(d_gpu[0].cpu(), d)
+    assert torch.equal(g_gpu[0].cpu().view(torch.int32), g.view(torch.int32))
+    L = gb.load_library()
+    r = gb.gac_result()
+    import ctypes
+    assert L.gac_stats(ctx.handle, 3, 0, None, ctypes.byref(r)) == gb.GAC_ERR_NONFINITE
+    gb.gac_free(ctx)
+
+
+def test_threshold_equality_is_inclusive_on_device():
+    """Exact-equality scalars through gac_decide: |c| == c_low is safe and
+    |c| == c_high is a violation (Algorithm 1)."""
+    g, d = [torch.ones(8, device="cuda")], [torch.ones(8, device="cuda")]
+    sums = torch.tensor([1.0, 4.0, 4.0], dtype=torch.float64, device="cuda")    # c = 0.25 exactly
+    scratch = torch.zeros(3, dtype=torch.float64, device="cuda")
+    for hp, want in [(gb.HParams(c_low=0.25, c_high=0.5, eps=0.0), gb.GAC_REGIME_SAFE),
+                     (gb.HParams(c_low=0.125, c_high=0.25, eps=0.0), gb.GAC_REGIME_VIOLATION),
+                     (gb.HParams(c_low=0.125, c_high=0.5, eps=0.0), gb.GAC_REGIME_PROJECT)]:
+        ctx = gb.gac_init(g, d, hp)
+        gb.gac_stats_partial(ctx, 2, scratch)
+        res = gb.gac_decide(ctx, sums)
+        assert res.cos == 0.25 and res.regime == want
+        dec = orc.decide((1.0, 4.0, 4.0), to_orc_hp(hp))
+        assert (res.alpha, res.coef64, res.coef) == (dec.alpha, dec.coef64, dec.coef)
+        gb.gac_free(ctx)
+
+
+# --------------------------------------------------- determinism, sharded form
+
+def test_stats_are_bitwise_reproducible():
+    shapes = synth.decoder_tensor_list(synth.DIMS["small"])
+    g, d = synth.gradient_list(shapes, 0.3, config_id=2, device="cuda")
+    ctx = gb.gac_init(g, d, gb.HParams())
+    first = None
+    for _ in range(10):
+        r = gb.gac_stats(ctx, 2)
+        key = (r.dot, r.gg, r.dd, r.cos)
+        first = first or key
+        assert key == first
+    gb.gac_free(ctx)
+
+
+def test_sharded_partial_sums_add_up_to_the_whole():
+    """App. A.1: per-shard inner products, one sum of three numbers, same decision."""
+    shapes = synth.decoder_tensor_list(synth.DIMS["small"])
+    g, d = synth.gradient_list(shapes, 0.2, config_id=2, device="cuda")
+    hp = gb.HParams(**FORCE)
+    whole = gb.gac_init(g, d, hp)
+    ref = gb.gac_stats(whole, 2)
+    cut = len(g) // 2
+    parts = [gb.gac_init(g[:cut], d[:cut], hp), gb.gac_init(g[cut:], d[cut:], hp)]
+    bufs = [torch.zeros(3, dtype=torch.float64, device="cuda") for _ in parts]
+    for c, b in zip(parts, bufs):
+        gb.gac_stats_partial(c, 2, b)
+    total = bufs[0] + bufs[1]            # stands for the all-reduce
+    results = [gb.gac_decide(c, total) for c in parts]
+    for r in results:
+        assert abs(r.dot - ref.dot) <= 1e-12 * abs(ref.dot)
+        assert abs(r.gg - ref.gg) <= 1e-12 * ref.gg and abs(r.dd - ref.dd) <= 1e-12 * ref.dd
+        assert r.regime == ref.regime
+    assert results[0].coef == results[1].coef and results[0].cos == results[1].cos
+    g_ref = [t.cpu() for t in g]
+    d_ref = [t.cpu() for t in d]
+    dec = orc.decide(orc.stats(g_ref, d_ref), to_orc_hp(hp))
+    orc.project(g_ref, d_ref, to_orc_hp(hp), dec)
+    for c in parts:
+        gb.gac_project(c, coef_override=dec.coef)
+    torch.cuda.synchronize()
+    check_outputs(g, d, g_ref, d_ref)
+    for c in parts + [whole]:
+        gb.gac_free(c)
+
+
+def test_call_order_is_enforced():
+    g, d = [torch.ones(100, device="cuda")], [torch.ones(100, device="cuda") * 2]
+    ctx = gb.gac_init(g, d, gb.HParams())
+    with pytest.raises(gb.GacError) as e:
+        gb.gac_project(ctx)
+    assert e.value.status == gb.GAC_ERR_STATE
+    with pytest.raises(gb.GacError) as e:
+        gb.gac_stats(ctx, 0)
+    assert e.value.status == gb.GAC_ERR_INVALID_ARG
+    gb.gac_stats(ctx, 5)
+    gb.gac_project(ctx)
+    with pytest.raises(gb.GacError) as e:
+        gb.gac_project(ctx)
+    assert e.value.status == gb.GAC_ERR_STATE
+    with pytest.raises(gb.GacError) as e:
+        gb.gac_stats(ctx, 5)
+    assert e.value.status == gb.GAC_ERR_STATE
+    gb.gac_stats(ctx, 6)
+    info = gb.gac_get_info(ctx)
+    assert info.launches == 3 and info.total_elems == 100
+    gb.gac_free(ctx)
