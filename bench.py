@@ -60,7 +60,7 @@ class ClockSampler:
     """Samples SM clock and throttle reasons through NVML (read-only) while the
     timed region runs."""
 
-    def __init__(self, index: int, period_s: float = 0.1):
+    def __init__(self, index: int, period_s: float = 0.02):
         self.index, self.period = index, period_s
         self.samples, self.reasons, self.max_mhz = [], set(), None
         self._stop = threading.Event()
@@ -475,7 +475,9 @@ def main():
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         probe = time_oracle(args.workload, 8_000_000, 1, 0)
         target = int(min(1_500_000_000, max(8_000_000, probe["value"] * 6.0)))
-        cb = time_oracle(args.workload, target, 2, 1)
+        first = time_oracle(args.workload, target, 1, 1)
+        passes = int(min(30, max(2, math.ceil(12.0 / max(first["seconds_per_pass"], 1e-3)))))
+        cb = time_oracle(args.workload, target, passes, 0)
         line["cpu_baseline"] = {k: cb[k] for k in ("value", "unit", "cores", "kind", "sample")}
 
     if world > 1:

@@ -359,6 +359,7 @@ __device__ __forceinline__ void project_chunk(const Chunk &ch, float k, double b
                 const uint32_t v = base + u * kThreads + tid;
                 if (v >= nvec) continue;
                 F4 out = gv[u];
+                if (GOP == G_ZERO) out = F4{0.f, 0.f, 0.f, 0.f};
                 if (GOP == G_FMA) {
                     out.x = rank_one<BETA1>(gv[u].x, dv[u].x, k, beta);
                     out.y = rank_one<BETA1>(gv[u].y, dv[u].y, k, beta);
@@ -377,7 +378,7 @@ __device__ __forceinline__ void project_chunk(const Chunk &ch, float k, double b
         if (tid < ch.n - done) {
             const uint32_t i = done + tid;
             const float x = kReadG ? Elem<GT>::load1(g, i) : 0.f;
-            float out = x;
+            float out = (GOP == G_ZERO) ? 0.f : x;
             if (GOP == G_FMA) out = rank_one<BETA1>(x, Elem<float>::load1(d, i), k, beta);
             if (GOP != G_KEEP) Elem<GT>::store1(g, i, out);
             if (DOP == D_RAW) Elem<float>::store1(d, i, x);
@@ -389,7 +390,7 @@ __device__ __forceinline__ void project_chunk(const Chunk &ch, float k, double b
     } else {
         for (uint32_t i = tid; i < ch.n; i += kThreads) {
             const float x = kReadG ? Elem<GT>::load1(g, i) : 0.f;
-            float out = x;
+            float out = (GOP == G_ZERO) ? 0.f : x;
             if (GOP == G_FMA) out = rank_one<BETA1>(x, Elem<float>::load1(d, i), k, beta);
             if (GOP != G_KEEP) Elem<GT>::store1(g, i, out);
             if (DOP == D_RAW) Elem<float>::store1(d, i, x);

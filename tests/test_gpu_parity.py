@@ -171,7 +171,8 @@ def test_variants(hp, g_dtype):
     res, dec, gg, dg, gr, dr = step_both([g], [d], hp)
     check_sums(res, dec)
     check_decision(res, dec)
-    check_outputs(gg, dg, gr, dr)
+    follows = hp.state_mode == gb.GAC_STATE_PROJECTED and res.regime == gb.GAC_REGIME_PROJECT
+    check_outputs(gg, dg, gr, dr, d_follows_g=follows)
 
 
 def test_degenerate_vectors():
