@@ -41,6 +41,8 @@ DIMS: Dict[str, DecoderDims] = {
     "14b": DecoderDims(5120, 48, 40, 8, 128, 13824, 152064, False),
     # scaled-down lists with the same structure, for cases a CPU checks in seconds;
     # odd sizes on purpose so tensor tails are ragged
+    # a 0.25 B list (1-2 GB per buffer): larger than L2, small enough for profiler captures
+    "0.25b": DecoderDims(1024, 12, 8, 2, 128, 4096, 32000, False),
     "mini": DecoderDims(96, 3, 3, 1, 32, 250, 1021, True),
     "small": DecoderDims(384, 6, 6, 2, 64, 1030, 15013, False),
 }
@@ -215,6 +217,8 @@ WORKLOADS = {
     "cfg2_1.5b_f32": ("1.5b", torch.float32, 0.8, 2),
     "cfg3_7b_bf16": ("7b", torch.bfloat16, 0.95, 3),
     "cfg5_14b_f32": ("14b", torch.float32, 0.9, 5),
+    "prof_0.25b_f32": ("0.25b", torch.float32, 0.9, 5),
+    "prof_0.25b_bf16": ("0.25b", torch.bfloat16, 0.95, 3),
     "small_f32": ("small", torch.float32, 0.9, 2),
     "small_bf16": ("small", torch.bfloat16, 0.95, 3),
 }
