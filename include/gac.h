@@ -195,6 +195,54 @@ typedef struct {
 } gac_info;
 int gac_get_info(const gac_ctx *ctx, gac_info *out);
 
+/*
+ * gac_stats_static -- gac_stats for callers that must not allocate.
+ * (No counterpart in the paper: it computes exactly what gac_stats computes;
+ * only where the work memory comes from differs.)
+ *
+ * Who needs it: code that runs where asking the driver for device memory is
+ * off limits -- inside a region whose memory is wholly owned by a framework's
+ * pool (so a cudaMalloc could fail or fragment it), on a latency-critical path
+ * where the implicit device-wide synchronisation of cudaMalloc/cudaFree is
+ * unacceptable, or in a process that was told to keep a fixed memory footprint.
+ * gac_init allocates a chunk table, partial sums and a pinned mirror; this
+ * entry point needs no context and calls no allocating CUDA routine at all.
+ *
+ * How: the chunk table, the per-CTA partial sums and the arrival ticket live
+ * in an array that is part of the library image: GAC_STATIC_SCRATCH_BYTES
+ * (about 2.1 MiB) on EVERY device that loads the library, held until the
+ * process exits.  The list is cut into chunks of 16384 elements, none spanning
+ * two tensors; at most GAC_STATIC_MAX_CHUNKS chunks fit (65536: up to about
+ * 1.07e9 elements; every tensor costs at least one chunk).  A list that needs
+ * more is refused with GAC_ERR_INVALID_ARG and a message; use gac_init then.
+ *
+ *   list, n, g_dtype, d_dtype, hp, step, staleness   as in gac_init / gac_stats
+ *                    (list is a host pointer; g and d inside are device
+ *                    pointers, caller-owned, only read)
+ *   cuda_device      device that owns g, d and result_dev (0..63)
+ *   cuda_stream      stream for the two small copies and the one kernel launch
+ *   result_dev       DEVICE pointer, caller-owned: receives the gac_result of
+ *                    this step when the stream reaches that point.  Nothing is
+ *                    copied to the host and the call does not synchronise.
+ *
+ * The first call on each device looks up the device address of the built-in
+ * array (once, with that device current); make that first call outside any
+ * stream capture.  Later calls reuse the address.
+ *
+ * All calls on a device share the one array, and it keeps what the previous
+ * call left: each call re-zeroes the ticket and rewrites the table on its
+ * stream before launching.  Two calls whose GPU work overlaps (different
+ * streams without ordering, or two host threads) race on that array and give
+ * wrong sums: order them on one stream or with events.
+ * Only the statistics pass has this form; gac_project still wants a context.
+ * Errors: INVALID_ARG, DTYPE, CUDA (message via gac_last_error(NULL)).
+ */
+#define GAC_STATIC_MAX_CHUNKS 65536
+#define GAC_STATIC_SCRATCH_BYTES (256 + 62976 + GAC_STATIC_MAX_CHUNKS * 32)
+int gac_stats_static(const gac_tensor *list, uint32_t n, int g_dtype, int d_dtype,
+                     const gac_hparams *hp, uint64_t step, uint32_t staleness, int cuda_device,
+                     void *cuda_stream, gac_result *result_dev);
+
 #ifdef __cplusplus
 }
 #endif

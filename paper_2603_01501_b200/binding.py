@@ -55,7 +55,8 @@ class gac_info(ctypes.Structure):
 
 
 EXPORTS = ["gac_default_hparams", "gac_init", "gac_stats", "gac_stats_partial", "gac_decide",
-           "gac_project", "gac_free", "gac_last_error", "gac_set_launch", "gac_get_info"]
+           "gac_project", "gac_free", "gac_last_error", "gac_set_launch", "gac_get_info",
+           "gac_stats_static"]
 
 _lib = None
 
@@ -90,6 +91,9 @@ def load_library() -> ctypes.CDLL:
     L.gac_last_error.restype = ctypes.c_char_p
     L.gac_set_launch.argtypes = [vp, i32, i32]
     L.gac_get_info.argtypes = [vp, ctypes.POINTER(gac_info)]
+    L.gac_stats_static.argtypes = [ctypes.POINTER(gac_tensor), u32, i32, i32,
+                                   ctypes.POINTER(gac_hparams), u64, u32, i32, vp, vp]
+    L.gac_stats_static.restype = i32
     for name in ("gac_init", "gac_stats", "gac_stats_partial", "gac_decide", "gac_project",
                  "gac_free", "gac_set_launch", "gac_get_info"):
         getattr(L, name).restype = i32
@@ -232,3 +236,34 @@ def gac_get_info(ctx: GacContext) -> gac_info:
     info = gac_info()
     ctx._check(load_library().gac_get_info(ctx.handle, ctypes.byref(info)))
     return info
+
+
+def gac_stats_static(g_list: Sequence[torch.Tensor], d_list: Sequence[torch.Tensor], hp: HParams,
+                     step: int, result_dev: torch.Tensor, staleness: int = 0, stream=None) -> None:
+    """gac_stats_static of the C ABI: the statistics and the decision of one step
+    without any allocation by the library (work memory is built into it).
+    `result_dev` is a caller-owned CUDA uint8 tensor of at least
+    ``ctypes.sizeof(gac_result)`` bytes that receives the record on the stream;
+    read it with ``result_from_tensor`` after synchronising."""
+    L = load_library()
+    if not (result_dev.is_cuda and result_dev.dtype == torch.uint8 and result_dev.is_contiguous()
+            and result_dev.numel() >= ctypes.sizeof(gac_result) and result_dev.data_ptr() % 8 == 0):
+        raise ValueError("result_dev must be an 8-byte aligned CUDA uint8 tensor of >= 72 bytes")
+    n = len(g_list)
+    arr = (gac_tensor * max(n, 1))()
+    for i, (g, d) in enumerate(zip(g_list, d_list)):
+        arr[i] = gac_tensor(g.data_ptr(), d.data_ptr(), g.numel())
+    chp = hp.c()
+    g_dt = _DT[g_list[0].dtype] if n else 0
+    d_dt = _DT[d_list[0].dtype] if n else 0
+    dev = result_dev.device.index
+    rc = L.gac_stats_static(arr, n, g_dt, d_dt, ctypes.byref(chp), step, staleness, dev,
+                            _stream_ptr(stream), result_dev.data_ptr())
+    if rc != GAC_OK:
+        raise GacError(rc, L.gac_last_error(None).decode())
+
+
+def result_from_tensor(t: torch.Tensor) -> gac_result:
+    """Decodes a gac_result held in a uint8 tensor (copied to the host here)."""
+    raw = bytes(t.detach().cpu().numpy().tobytes()[: ctypes.sizeof(gac_result)])
+    return gac_result.from_buffer_copy(raw)

@@ -22,6 +22,7 @@
 #include <string.h>
 
 #include <algorithm>
+#include <mutex>
 #include <new>
 #include <vector>
 
@@ -820,3 +821,133 @@ int gac_get_info(const gac_ctx *ctx, gac_info *out) {
 }
 
 }  // extern "C"
+
+// ------------------------------------------------ allocation-free statistics
+//
+// Everything gac_stats needs beyond its inputs and outputs -- the chunk table,
+// the per-CTA partial sums and the arrival ticket -- laid out in one array that
+// is part of the loaded library image, so that no call ever has to ask the
+// driver for device memory.  Every device that loads the library carries its
+// own copy (about 2.1 MiB) until the process exits.
+namespace {
+
+constexpr uint32_t kStaticMaxChunks = GAC_STATIC_MAX_CHUNKS;
+constexpr uint32_t kStaticMaxCtas = 148 * 16 + 256;             // grid never exceeds SMs x resident CTAs
+constexpr size_t kStaticTicketOff = 0;                           // one unsigned, rest of the 256 bytes unused
+constexpr size_t kStaticPartialsOff = 256;
+constexpr size_t kStaticChunksOff = kStaticPartialsOff + ((size_t(kStaticMaxCtas) * 3 * sizeof(double) + 255) / 256) * 256;
+constexpr size_t kStaticBytes = kStaticChunksOff + size_t(kStaticMaxChunks) * sizeof(Chunk);
+static_assert(kStaticBytes == GAC_STATIC_SCRATCH_BYTES, "the header states the size of the built-in scratch");
+
+static __device__ __align__(256) unsigned char g_static_scratch[kStaticBytes];
+
+constexpr int kMaxDevices = 64;
+struct StaticSetup {
+    bool ready = false;
+    unsigned char *base = nullptr;   // DEVICE address of g_static_scratch on that device
+    int sms = 0;
+    int occ_f32 = 0, occ_bf16 = 0;
+};
+StaticSetup g_static_setup[kMaxDevices];
+std::mutex g_static_mutex;
+
+// Runs once per device, with that device current.  The array's name is only a
+// host-side handle here; the address a kernel can use comes from the runtime.
+int static_setup(int dev, StaticSetup **out) {
+    std::lock_guard<std::mutex> lock(g_static_mutex);
+    StaticSetup &st = g_static_setup[dev];
+    if (!st.ready) {
+        void *ptr = nullptr;
+        cudaError_t e = cudaGetSymbolAddress(&ptr, g_static_scratch);
+        if (e != cudaSuccess || !ptr)
+            return fail(nullptr, GAC_ERR_CUDA, "cudaGetSymbolAddress failed: %s (CUDA error %lld)",
+                        cudaGetErrorString(e), (long long)e);
+        e = cudaDeviceGetAttribute(&st.sms, cudaDevAttrMultiProcessorCount, dev);
+        if (e != cudaSuccess)
+            return fail(nullptr, GAC_ERR_CUDA, "cudaDeviceGetAttribute failed: %s (CUDA error %lld)",
+                        cudaGetErrorString(e), (long long)e);
+        st.occ_f32 = resident_ctas(gac_stats_kernel<float>);
+        st.occ_bf16 = resident_ctas(gac_stats_kernel<bf16_t>);
+        st.base = static_cast<unsigned char *>(ptr);
+        st.ready = true;
+    }
+    *out = &st;
+    return GAC_OK;
+}
+
+}  // namespace
+
+extern "C" int gac_stats_static(const gac_tensor *list, uint32_t n, int g_dtype, int d_dtype,
+                                const gac_hparams *hp, uint64_t step, uint32_t staleness,
+                                int cuda_device, void *cuda_stream, gac_result *result_dev) {
+    if (!list || n == 0) return fail(nullptr, GAC_ERR_INVALID_ARG, "empty tensor list%s");
+    if (!hp) return fail(nullptr, GAC_ERR_INVALID_ARG, "hp is NULL%s");
+    if (!result_dev) return fail(nullptr, GAC_ERR_INVALID_ARG, "result_dev is NULL%s");
+    if (step == 0) return fail(nullptr, GAC_ERR_INVALID_ARG, "step counts from 1 (Algorithm 1)%s");
+    if (!((g_dtype == GAC_F32 || g_dtype == GAC_BF16) && d_dtype == GAC_F32))
+        return fail(nullptr, GAC_ERR_DTYPE, "supported (g,d) element types: (f32,f32), (bf16,f32)%s");
+    if (int rc = check_hparams(hp)) return rc;
+    if (cuda_device < 0 || cuda_device >= kMaxDevices)
+        return fail(nullptr, GAC_ERR_INVALID_ARG, "cuda_device %s%lld out of range", "", cuda_device);
+
+    // count the chunks first and refuse what does not fit the built-in scratch
+    const uint64_t ce = kDefaultChunk;
+    const size_t gs = elem_size(g_dtype), ds = elem_size(d_dtype);
+    uint64_t n_chunks = 0;
+    for (uint32_t i = 0; i < n; ++i) {
+        if (!list[i].g || !list[i].d || list[i].numel == 0)
+            return fail(nullptr, GAC_ERR_INVALID_ARG, "tensor %s%lld has a NULL pointer or no elements", "", i);
+        if (reinterpret_cast<uint64_t>(list[i].g) % gs || reinterpret_cast<uint64_t>(list[i].d) % ds)
+            return fail(nullptr, GAC_ERR_INVALID_ARG, "tensor %s%lld is not element-aligned", "", i);
+        n_chunks += (list[i].numel + ce - 1) / ce;
+        if (n_chunks > kStaticMaxChunks)
+            return fail(nullptr, GAC_ERR_INVALID_ARG,
+                        "list needs more than %s%lld chunks of 16384 elements: beyond the built-in scratch; "
+                        "use gac_init/gac_stats", "", (long long)kStaticMaxChunks);
+    }
+
+    DeviceGuard guard(cuda_device);
+    if (!guard.ok) return fail(nullptr, GAC_ERR_CUDA, "cudaSetDevice failed%s");
+    StaticSetup *st = nullptr;
+    if (int rc = static_setup(cuda_device, &st)) return rc;
+
+    // host-side image of the table (host memory only), then one copy into the scratch
+    static thread_local std::vector<Chunk> table;
+    table.clear();
+    table.reserve(n_chunks);
+    for (uint32_t i = 0; i < n; ++i) {
+        const uint64_t gb = reinterpret_cast<uint64_t>(list[i].g), db = reinterpret_cast<uint64_t>(list[i].d);
+        const bool aligned = (gb % 16 == 0) && (db % 16 == 0);
+        for (uint64_t off = 0; off < list[i].numel; off += ce) {
+            Chunk ch;
+            ch.g = gb + off * gs;
+            ch.d = db + off * ds;
+            ch.n = uint32_t(std::min<uint64_t>(ce, list[i].numel - off));
+            ch.flags = aligned ? kChunkAligned : 0u;
+            ch.pad = 0;
+            table.push_back(ch);
+        }
+    }
+    cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+    Chunk *d_chunks = reinterpret_cast<Chunk *>(st->base + kStaticChunksOff);
+    double *d_partials = reinterpret_cast<double *>(st->base + kStaticPartialsOff);
+    unsigned *d_ticket = reinterpret_cast<unsigned *>(st->base + kStaticTicketOff);
+    // the scratch keeps whatever the previous call left: the ticket must start at zero
+    GAC_CUDA(nullptr, cudaMemsetAsync(d_ticket, 0, sizeof(unsigned), s));
+    // source is pageable host memory: the call returns once it has been staged, so `table` may be reused
+    GAC_CUDA(nullptr, cudaMemcpyAsync(d_chunks, table.data(), table.size() * sizeof(Chunk),
+                                      cudaMemcpyHostToDevice, s));
+    gac_ctx shell;            // only carries the hyper-parameters into dev_hp()
+    shell.hp = *hp;
+    const DevHP h = dev_hp(&shell, step, staleness, 1);
+    const int occ = g_dtype == GAC_BF16 ? st->occ_bf16 : st->occ_f32;
+    const uint32_t grid = uint32_t(std::min<uint64_t>(std::min<uint64_t>(uint64_t(st->sms) * occ, kStaticMaxCtas), n_chunks));
+    if (g_dtype == GAC_BF16)
+        gac_stats_kernel<bf16_t><<<grid, kThreads, 0, s>>>(d_chunks, uint32_t(n_chunks), d_partials, d_ticket,
+                                                           result_dev, nullptr, h);
+    else
+        gac_stats_kernel<float><<<grid, kThreads, 0, s>>>(d_chunks, uint32_t(n_chunks), d_partials, d_ticket,
+                                                          result_dev, nullptr, h);
+    GAC_CUDA(nullptr, cudaGetLastError());
+    return GAC_OK;
+}
