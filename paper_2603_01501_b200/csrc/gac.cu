@@ -30,10 +30,77 @@
 
 namespace {
 
-constexpr int kThreads = 256;        // threads per CTA in both kernels
-constexpr int kUnroll = 4;           // 4-element vectors in flight per thread and operand
-constexpr int kDefaultChunk = 16384; // elements per chunk
-constexpr int kMaxCtasPerSm = 8;
+// Launch geometry.  Both kernels are bound by HBM, and on B200 their speed
+// depends on how many bytes each SM keeps in flight: too few starve the
+// memory system, too many make reads and write-backs of many chunks collide in
+// DRAM.  The macros exist so that variants can be built and timed side by side;
+// the defaults are the measured best per element type (T threads per CTA,
+// U four-element vectors in flight per thread and operand, C resident CTAs per
+// SM the grid is sized for with 0 = all that fit, MINB = occupancy asked of the
+// compiler with 0 = no request).
+#ifndef GAC_STATS_T_F32
+#define GAC_STATS_T_F32 256
+#endif
+#ifndef GAC_STATS_U_F32
+#define GAC_STATS_U_F32 8
+#endif
+#ifndef GAC_STATS_C_F32
+#define GAC_STATS_C_F32 0
+#endif
+#ifndef GAC_STATS_MINB_F32
+#define GAC_STATS_MINB_F32 4
+#endif
+#ifndef GAC_STATS_T_BF16
+#define GAC_STATS_T_BF16 256
+#endif
+#ifndef GAC_STATS_U_BF16
+#define GAC_STATS_U_BF16 8
+#endif
+#ifndef GAC_STATS_C_BF16
+#define GAC_STATS_C_BF16 0
+#endif
+#ifndef GAC_STATS_MINB_BF16
+#define GAC_STATS_MINB_BF16 4
+#endif
+#ifndef GAC_PROJ_T_F32
+#define GAC_PROJ_T_F32 256
+#endif
+#ifndef GAC_PROJ_U_F32
+#define GAC_PROJ_U_F32 8
+#endif
+#ifndef GAC_PROJ_C_F32
+#define GAC_PROJ_C_F32 1
+#endif
+#ifndef GAC_PROJ_MINB_F32
+#define GAC_PROJ_MINB_F32 1
+#endif
+#ifndef GAC_PROJ_T_BF16
+#define GAC_PROJ_T_BF16 512
+#endif
+#ifndef GAC_PROJ_U_BF16
+#define GAC_PROJ_U_BF16 4
+#endif
+#ifndef GAC_PROJ_C_BF16
+#define GAC_PROJ_C_BF16 1
+#endif
+#ifndef GAC_PROJ_MINB_BF16
+#define GAC_PROJ_MINB_BF16 1
+#endif
+#ifndef GAC_CHUNK
+#define GAC_CHUNK 16384
+#endif
+// load flavour: 0 plain ld.global, 1 streaming (ld.global.cs), 2 read-only path (ld.global.nc)
+#ifndef GAC_LD_STATS
+#define GAC_LD_STATS 0
+#endif
+#ifndef GAC_LD_PROJECT
+#define GAC_LD_PROJECT 0
+#endif
+#ifndef GAC_ST      // 0 plain st.global, 1 streaming (st.global.cs), 2 write-through (st.global.wt)
+#define GAC_ST 1
+#endif
+constexpr int kDefaultChunk = GAC_CHUNK; // elements per chunk
+constexpr int kMaxCtasPerSm = 16;
 
 constexpr uint32_t kChunkAligned = 1u;  // both bases 16-byte aligned: vector path
 
@@ -61,17 +128,35 @@ struct F4 {
 
 // ---------------------------------------------------------------- element I/O
 
+template <int LD, typename V>
+__device__ __forceinline__ V ld_vec(const V *p) {
+    if (LD == 1) return __ldcs(p);
+    if (LD == 2) return __ldg(p);
+    return *p;
+}
+template <typename V>
+__device__ __forceinline__ void st_vec(V *p, V v) {
+#if GAC_ST == 1
+    __stcs(p, v);
+#elif GAC_ST == 2
+    __stwt(p, v);
+#else
+    *p = v;
+#endif
+}
+
 template <typename GT>
 struct Elem;
 
 template <>
 struct Elem<float> {
+    template <int LD>
     static __device__ __forceinline__ F4 load4(const void *base, uint32_t v) {
-        float4 t = reinterpret_cast<const float4 *>(base)[v];
+        float4 t = ld_vec<LD>(reinterpret_cast<const float4 *>(base) + v);
         return F4{t.x, t.y, t.z, t.w};
     }
     static __device__ __forceinline__ void store4(void *base, uint32_t v, F4 a) {
-        reinterpret_cast<float4 *>(base)[v] = make_float4(a.x, a.y, a.z, a.w);
+        st_vec(reinterpret_cast<float4 *>(base) + v, make_float4(a.x, a.y, a.z, a.w));
     }
     static __device__ __forceinline__ float load1(const void *base, uint32_t i) {
         return reinterpret_cast<const float *>(base)[i];
@@ -86,6 +171,27 @@ struct bf16_t {
     uint16_t bits;
 };
 
+template <typename GT>
+struct StatsGeom;
+template <>
+struct StatsGeom<float> {
+    static constexpr int T = GAC_STATS_T_F32, U = GAC_STATS_U_F32, C = GAC_STATS_C_F32, MINB = GAC_STATS_MINB_F32;
+};
+template <>
+struct StatsGeom<bf16_t> {
+    static constexpr int T = GAC_STATS_T_BF16, U = GAC_STATS_U_BF16, C = GAC_STATS_C_BF16, MINB = GAC_STATS_MINB_BF16;
+};
+template <typename GT>
+struct ProjGeom;
+template <>
+struct ProjGeom<float> {
+    static constexpr int T = GAC_PROJ_T_F32, U = GAC_PROJ_U_F32, C = GAC_PROJ_C_F32, MINB = GAC_PROJ_MINB_F32;
+};
+template <>
+struct ProjGeom<bf16_t> {
+    static constexpr int T = GAC_PROJ_T_BF16, U = GAC_PROJ_U_BF16, C = GAC_PROJ_C_BF16, MINB = GAC_PROJ_MINB_BF16;
+};
+
 __device__ __forceinline__ uint32_t pack_bf16x2_rn(float lo, float hi) {
     uint32_t r;
     asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
@@ -94,14 +200,15 @@ __device__ __forceinline__ uint32_t pack_bf16x2_rn(float lo, float hi) {
 
 template <>
 struct Elem<bf16_t> {
+    template <int LD>
     static __device__ __forceinline__ F4 load4(const void *base, uint32_t v) {
-        uint2 t = reinterpret_cast<const uint2 *>(base)[v];
+        uint2 t = ld_vec<LD>(reinterpret_cast<const uint2 *>(base) + v);
         return F4{__uint_as_float(t.x << 16), __uint_as_float(t.x & 0xFFFF0000u),
                   __uint_as_float(t.y << 16), __uint_as_float(t.y & 0xFFFF0000u)};
     }
     static __device__ __forceinline__ void store4(void *base, uint32_t v, F4 a) {
-        reinterpret_cast<uint2 *>(base)[v] =
-            make_uint2(pack_bf16x2_rn(a.x, a.y), pack_bf16x2_rn(a.z, a.w));
+        st_vec(reinterpret_cast<uint2 *>(base) + v,
+               make_uint2(pack_bf16x2_rn(a.x, a.y), pack_bf16x2_rn(a.z, a.w)));
     }
     static __device__ __forceinline__ float load1(const void *base, uint32_t i) {
         return __uint_as_float(uint32_t(reinterpret_cast<const uint16_t *>(base)[i]) << 16);
@@ -182,6 +289,7 @@ __device__ __forceinline__ double warp_sum(double v) {
 }
 
 // Sums (a, b, c) over the CTA in a fixed order; the result is valid in thread 0.
+template <int T>
 __device__ __forceinline__ void block_sum3(double &a, double &b, double &c, double (*sm)[3]) {
     a = warp_sum(a);
     b = warp_sum(b);
@@ -197,7 +305,7 @@ __device__ __forceinline__ void block_sum3(double &a, double &b, double &c, doub
         a = sm[0][0];
         b = sm[0][1];
         c = sm[0][2];
-        for (int w = 1; w < kThreads / 32; ++w) {
+        for (int w = 1; w < T / 32; ++w) {
             a += sm[w][0];
             b += sm[w][1];
             c += sm[w][2];
@@ -212,23 +320,24 @@ __device__ __forceinline__ void stats_chunk(const Chunk &ch, double &a_dot, doub
     const void *g = reinterpret_cast<const void *>(ch.g);
     const void *d = reinterpret_cast<const void *>(ch.d);
     const uint32_t tid = threadIdx.x;
+    constexpr int T = StatsGeom<GT>::T, U = StatsGeom<GT>::U;
     if (ch.flags & kChunkAligned) {
         const uint32_t nvec = ch.n >> 2;
-        for (uint32_t base = 0; base < nvec; base += kThreads * kUnroll) {
-            F4 gv[kUnroll], dv[kUnroll];
+        for (uint32_t base = 0; base < nvec; base += T * U) {
+            F4 gv[U], dv[U];
 #pragma unroll
-            for (int u = 0; u < kUnroll; ++u) {
-                const uint32_t v = base + u * kThreads + tid;
+            for (int u = 0; u < U; ++u) {
+                const uint32_t v = base + u * T + tid;
                 if (v < nvec) {
-                    gv[u] = Elem<GT>::load4(g, v);
-                    if (READ_D) dv[u] = Elem<float>::load4(d, v);
+                    gv[u] = Elem<GT>::template load4<GAC_LD_STATS>(g, v);
+                    if (READ_D) dv[u] = Elem<float>::load4<GAC_LD_STATS>(d, v);
                 } else {
                     gv[u] = F4{0.f, 0.f, 0.f, 0.f};
                     if (READ_D) dv[u] = F4{0.f, 0.f, 0.f, 0.f};
                 }
             }
 #pragma unroll
-            for (int u = 0; u < kUnroll; ++u) {
+            for (int u = 0; u < U; ++u) {
                 const float ge[4] = {gv[u].x, gv[u].y, gv[u].z, gv[u].w};
                 const float de[4] = {dv[u].x, dv[u].y, dv[u].z, dv[u].w};
 #pragma unroll
@@ -254,7 +363,7 @@ __device__ __forceinline__ void stats_chunk(const Chunk &ch, double &a_dot, doub
             }
         }
     } else {   // a base that is not 16-byte aligned: element-wise, still coalesced
-        for (uint32_t i = tid; i < ch.n; i += kThreads) {
+        for (uint32_t i = tid; i < ch.n; i += T) {
             const double x = double(Elem<GT>::load1(g, i));
             a_gg = fma(x, x, a_gg);
             if (READ_D) {
@@ -270,10 +379,11 @@ __device__ __forceinline__ void stats_chunk(const Chunk &ch, double &a_dot, doub
 // ticket: zero on entry; the last CTA to arrive reduces the slots in index
 // order, publishes the result and puts the ticket back to zero.  No CTA waits.
 template <typename GT>
-__global__ void __launch_bounds__(kThreads)
+__global__ void __launch_bounds__(StatsGeom<GT>::T, StatsGeom<GT>::MINB)
 gac_stats_kernel(const Chunk *__restrict__ chunks, uint32_t n_chunks, double *partials,
                  unsigned *ticket, gac_result *rec, double *sums_out, DevHP hp) {
-    __shared__ double sm[kThreads / 32][3];
+    constexpr int T = StatsGeom<GT>::T;
+    __shared__ double sm[T / 32][3];
     __shared__ bool is_last;
     double a_dot = 0.0, a_gg = 0.0, a_dd = 0.0;
     if (hp.first_step) {
@@ -283,7 +393,7 @@ gac_stats_kernel(const Chunk *__restrict__ chunks, uint32_t n_chunks, double *pa
         for (uint32_t c = blockIdx.x; c < n_chunks; c += gridDim.x)
             stats_chunk<GT, true>(load_chunk(chunks, c), a_dot, a_gg, a_dd);
     }
-    block_sum3(a_dot, a_gg, a_dd, sm);
+    block_sum3<T>(a_dot, a_gg, a_dd, sm);
     if (threadIdx.x == 0) {
         double *slot = partials + 3 * size_t(blockIdx.x);
         slot[0] = a_dot;
@@ -299,13 +409,13 @@ gac_stats_kernel(const Chunk *__restrict__ chunks, uint32_t n_chunks, double *pa
     // second stage: thread t adds slots t, t+T, t+2T, ... in that order, then the
     // same fixed tree as above
     double s0 = 0.0, s1 = 0.0, s2 = 0.0;
-    for (uint32_t b = threadIdx.x; b < gridDim.x; b += kThreads) {
+    for (uint32_t b = threadIdx.x; b < gridDim.x; b += T) {
         const double *slot = partials + 3 * size_t(b);
         s0 += __ldcg(slot + 0);
         s1 += __ldcg(slot + 1);
         s2 += __ldcg(slot + 2);
     }
-    block_sum3(s0, s1, s2, sm);
+    block_sum3<T>(s0, s1, s2, sm);
     if (threadIdx.x == 0) {
         *ticket = 0u;
         if (sums_out) {
@@ -339,25 +449,26 @@ __device__ __forceinline__ void project_chunk(const Chunk &ch, float k, double b
     void *g = reinterpret_cast<void *>(ch.g);
     void *d = reinterpret_cast<void *>(ch.d);
     const uint32_t tid = threadIdx.x;
+    constexpr int T = ProjGeom<GT>::T, U = ProjGeom<GT>::U;
     constexpr bool kReadG = (GOP == G_FMA) || (DOP == D_RAW);
     constexpr bool kReadD = (GOP == G_FMA);
     if (ch.flags & kChunkAligned) {
         const uint32_t nvec = ch.n >> 2;
-        for (uint32_t base = 0; base < nvec; base += kThreads * kUnroll) {
-            F4 gv[kUnroll], dv[kUnroll];
+        for (uint32_t base = 0; base < nvec; base += T * U) {
+            F4 gv[U], dv[U];
 #pragma unroll
-            for (int u = 0; u < kUnroll; ++u) {
-                const uint32_t v = base + u * kThreads + tid;
+            for (int u = 0; u < U; ++u) {
+                const uint32_t v = base + u * T + tid;
                 gv[u] = F4{0.f, 0.f, 0.f, 0.f};
                 dv[u] = F4{0.f, 0.f, 0.f, 0.f};
                 if (v < nvec) {
-                    if (kReadG) gv[u] = Elem<GT>::load4(g, v);
-                    if (kReadD) dv[u] = Elem<float>::load4(d, v);
+                    if (kReadG) gv[u] = Elem<GT>::template load4<GAC_LD_PROJECT>(g, v);
+                    if (kReadD) dv[u] = Elem<float>::load4<GAC_LD_PROJECT>(d, v);
                 }
             }
 #pragma unroll
-            for (int u = 0; u < kUnroll; ++u) {
-                const uint32_t v = base + u * kThreads + tid;
+            for (int u = 0; u < U; ++u) {
+                const uint32_t v = base + u * T + tid;
                 if (v >= nvec) continue;
                 F4 out = gv[u];
                 if (GOP == G_ZERO) out = F4{0.f, 0.f, 0.f, 0.f};
@@ -370,7 +481,7 @@ __device__ __forceinline__ void project_chunk(const Chunk &ch, float k, double b
                 if (GOP != G_KEEP) Elem<GT>::store4(g, v, out);
                 if (DOP == D_RAW) Elem<float>::store4(d, v, gv[u]);
                 if (DOP == D_NEW) {
-                    if (GOP == G_FMA) out = Elem<GT>::load4(g, v);   // the value as stored (rounded)
+                    if (GOP == G_FMA) out = Elem<GT>::template load4<GAC_LD_PROJECT>(g, v);   // the value as stored (rounded)
                     Elem<float>::store4(d, v, out);
                 }
             }
@@ -389,7 +500,7 @@ __device__ __forceinline__ void project_chunk(const Chunk &ch, float k, double b
             }
         }
     } else {
-        for (uint32_t i = tid; i < ch.n; i += kThreads) {
+        for (uint32_t i = tid; i < ch.n; i += T) {
             const float x = kReadG ? Elem<GT>::load1(g, i) : 0.f;
             float out = (GOP == G_ZERO) ? 0.f : x;
             if (GOP == G_FMA) out = rank_one<BETA1>(x, Elem<float>::load1(d, i), k, beta);
@@ -411,33 +522,38 @@ __device__ __forceinline__ void project_walk(const Chunk *chunks, uint32_t n_chu
 }
 
 // The regime is read from the device-resident record, so no host round trip
-// separates the two passes.  Every CTA takes the same (uniform) branch.
-template <typename GT>
-__global__ void __launch_bounds__(kThreads)
+// separates the two passes; every CTA takes the same (uniform) branch.  What
+// the host already knows (state mode, beta == 1, zero_on_violation) is fixed at
+// compile time so that each instantiation holds only the loops it can reach.
+template <typename GT, int STATE, bool BETA1, bool ZERO>
+__global__ void __launch_bounds__(ProjGeom<GT>::T, ProjGeom<GT>::MINB)
 gac_project_kernel(const Chunk *__restrict__ chunks, uint32_t n_chunks, const gac_result *rec,
-                   float coef_override, int use_override, DevHP hp) {
+                   float coef_override, int use_override, double beta) {
     if (rec->nonfinite) return;   // reading taken for NaN/Inf: touch nothing
     const int regime = rec->regime;
     const float k = use_override ? coef_override : rec->coef;
-    int gop = G_KEEP;
-    if (regime == GAC_REGIME_PROJECT) gop = G_FMA;
-    else if (regime == GAC_REGIME_VIOLATION && hp.zero_on_violation) gop = G_ZERO;
-    int dop = D_KEEP;
-    if (hp.state_mode == GAC_STATE_RAW) dop = D_RAW;
-    else if (hp.state_mode == GAC_STATE_PROJECTED) dop = (gop == G_KEEP) ? D_RAW : D_NEW;
-    const bool beta1 = (hp.beta == 1.0);
+    constexpr int dop = STATE == GAC_STATE_RAW ? D_RAW : (STATE == GAC_STATE_PROJECTED ? D_NEW : D_KEEP);
+    if (regime == GAC_REGIME_PROJECT) {
+        project_walk<GT, G_FMA, dop, BETA1>(chunks, n_chunks, k, beta);
+    } else if (ZERO && regime == GAC_REGIME_VIOLATION) {
+        project_walk<GT, G_ZERO, dop, true>(chunks, n_chunks, k, 1.0);
+    } else if (STATE != GAC_STATE_HOLD) {
+        project_walk<GT, G_KEEP, D_RAW, true>(chunks, n_chunks, k, 1.0);   // d' = g, g untouched
+    }
+}
 
-    if (gop == G_FMA && dop == D_RAW && beta1) project_walk<GT, G_FMA, D_RAW, true>(chunks, n_chunks, k, 1.0);
-    else if (gop == G_KEEP && dop == D_RAW) project_walk<GT, G_KEEP, D_RAW, true>(chunks, n_chunks, k, 1.0);
-    else if (gop == G_KEEP && dop == D_KEEP) return;
-    else if (gop == G_FMA && dop == D_RAW) project_walk<GT, G_FMA, D_RAW, false>(chunks, n_chunks, k, hp.beta);
-    else if (gop == G_FMA && dop == D_NEW && beta1) project_walk<GT, G_FMA, D_NEW, true>(chunks, n_chunks, k, 1.0);
-    else if (gop == G_FMA && dop == D_NEW) project_walk<GT, G_FMA, D_NEW, false>(chunks, n_chunks, k, hp.beta);
-    else if (gop == G_FMA && dop == D_KEEP && beta1) project_walk<GT, G_FMA, D_KEEP, true>(chunks, n_chunks, k, 1.0);
-    else if (gop == G_FMA && dop == D_KEEP) project_walk<GT, G_FMA, D_KEEP, false>(chunks, n_chunks, k, hp.beta);
-    else if (gop == G_ZERO && dop == D_RAW) project_walk<GT, G_ZERO, D_RAW, true>(chunks, n_chunks, k, 1.0);
-    else if (gop == G_ZERO && dop == D_NEW) project_walk<GT, G_ZERO, D_NEW, true>(chunks, n_chunks, k, 1.0);
-    else if (gop == G_ZERO && dop == D_KEEP) project_walk<GT, G_ZERO, D_KEEP, true>(chunks, n_chunks, k, 1.0);
+using ProjectKernel = void (*)(const Chunk *, uint32_t, const gac_result *, float, int, double);
+
+template <typename GT, int STATE>
+ProjectKernel pick_project(bool beta1, bool zero) {
+    if (beta1) return zero ? gac_project_kernel<GT, STATE, true, true> : gac_project_kernel<GT, STATE, true, false>;
+    return zero ? gac_project_kernel<GT, STATE, false, true> : gac_project_kernel<GT, STATE, false, false>;
+}
+template <typename GT>
+ProjectKernel pick_project(int state, bool beta1, bool zero) {
+    if (state == GAC_STATE_RAW) return pick_project<GT, GAC_STATE_RAW>(beta1, zero);
+    if (state == GAC_STATE_PROJECTED) return pick_project<GT, GAC_STATE_PROJECTED>(beta1, zero);
+    return pick_project<GT, GAC_STATE_HOLD>(beta1, zero);
 }
 
 }  // namespace
@@ -463,6 +579,8 @@ struct gac_ctx {
     int chunk_elems = kDefaultChunk;
     int ctas_per_sm = 0;           // 0 = what occupancy allows
     int grid_stats = 0, grid_project = 0;
+    int threads_stats = 0, threads_project = 0;
+    const void *project_fn = nullptr;   // instantiation chosen from the hyper-parameters
 
     uint64_t last_projected_step = 0;
     uint64_t pending_step = 0;
@@ -520,9 +638,9 @@ void release_device(gac_ctx *c) {
 }
 
 template <typename K>
-int resident_ctas(K kernel) {
+int resident_ctas(K kernel, int threads) {
     int n = 0;
-    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, kernel, kThreads, 0) != cudaSuccess || n < 1)
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, kernel, threads, 0) != cudaSuccess || n < 1)
         n = 1;
     return std::min(n, kMaxCtasPerSm);
 }
@@ -562,10 +680,20 @@ int build_table(gac_ctx *c) {
                            cudaMemcpyHostToDevice));
     c->n_chunks = table.size();
 
-    int occ_s = c->g_dt == GAC_BF16 ? resident_ctas(gac_stats_kernel<bf16_t>)
-                                    : resident_ctas(gac_stats_kernel<float>);
-    int occ_p = c->g_dt == GAC_BF16 ? resident_ctas(gac_project_kernel<bf16_t>)
-                                    : resident_ctas(gac_project_kernel<float>);
+    const bool bf = (c->g_dt == GAC_BF16);
+    c->threads_stats = bf ? StatsGeom<bf16_t>::T : StatsGeom<float>::T;
+    c->threads_project = bf ? ProjGeom<bf16_t>::T : ProjGeom<float>::T;
+    int occ_s = bf ? resident_ctas(gac_stats_kernel<bf16_t>, c->threads_stats)
+                   : resident_ctas(gac_stats_kernel<float>, c->threads_stats);
+    const bool beta1 = (c->hp.beta == 1.0), zero = (c->hp.zero_on_violation != 0);
+    ProjectKernel pk = c->g_dt == GAC_BF16 ? pick_project<bf16_t>(c->hp.state_mode, beta1, zero)
+                                           : pick_project<float>(c->hp.state_mode, beta1, zero);
+    c->project_fn = reinterpret_cast<const void *>(pk);
+    int occ_p = resident_ctas(pk, c->threads_project);
+    const int cap_s = bf ? StatsGeom<bf16_t>::C : StatsGeom<float>::C;
+    const int cap_p = bf ? ProjGeom<bf16_t>::C : ProjGeom<float>::C;
+    if (cap_s > 0) occ_s = std::min(occ_s, cap_s);
+    if (cap_p > 0) occ_p = std::min(occ_p, cap_p);
     if (c->ctas_per_sm > 0) {
         occ_s = std::min(occ_s, c->ctas_per_sm);
         occ_p = std::min(occ_p, c->ctas_per_sm);
@@ -629,10 +757,10 @@ int launch_stats(gac_ctx *c, uint64_t step, uint32_t staleness, cudaStream_t s, 
     const DevHP h = dev_hp(c, step, staleness, decide);
     const uint32_t nc = uint32_t(c->n_chunks);
     if (c->g_dt == GAC_BF16)
-        gac_stats_kernel<bf16_t><<<c->grid_stats, kThreads, 0, s>>>(c->d_chunks, nc, c->d_partials,
+        gac_stats_kernel<bf16_t><<<c->grid_stats, c->threads_stats, 0, s>>>(c->d_chunks, nc, c->d_partials,
                                                                     c->d_ticket, c->d_rec, sums_out, h);
     else
-        gac_stats_kernel<float><<<c->grid_stats, kThreads, 0, s>>>(c->d_chunks, nc, c->d_partials,
+        gac_stats_kernel<float><<<c->grid_stats, c->threads_stats, 0, s>>>(c->d_chunks, nc, c->d_partials,
                                                                    c->d_ticket, c->d_rec, sums_out, h);
     GAC_CUDA(c, cudaGetLastError());
     ++c->launches;
@@ -779,14 +907,11 @@ int gac_project(gac_ctx *ctx, void *cuda_stream, const float *coef_override, gac
         return fail(ctx, GAC_ERR_STATE, "gac_project needs the decision of gac_stats / gac_decide for this step%s");
     DeviceGuard guard(ctx->device);
     cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
-    const DevHP h = dev_hp(ctx, ctx->pending_step, 0, 1);
     const float k = coef_override ? *coef_override : 0.0f;
     const int use = coef_override ? 1 : 0;
     const uint32_t nc = uint32_t(ctx->n_chunks);
-    if (ctx->g_dt == GAC_BF16)
-        gac_project_kernel<bf16_t><<<ctx->grid_project, kThreads, 0, s>>>(ctx->d_chunks, nc, ctx->d_rec, k, use, h);
-    else
-        gac_project_kernel<float><<<ctx->grid_project, kThreads, 0, s>>>(ctx->d_chunks, nc, ctx->d_rec, k, use, h);
+    reinterpret_cast<ProjectKernel>(const_cast<void *>(ctx->project_fn))<<<ctx->grid_project, ctx->threads_project, 0, s>>>(
+        ctx->d_chunks, nc, ctx->d_rec, k, use, ctx->hp.beta);
     GAC_CUDA(ctx, cudaGetLastError());
     ++ctx->launches;
     ctx->decision_ready = false;
@@ -812,7 +937,7 @@ int gac_get_info(const gac_ctx *ctx, gac_info *out) {
     out->n_chunks = ctx->n_chunks;
     out->n_tensors = uint32_t(ctx->list.size());
     out->grid = uint32_t(ctx->grid_stats);
-    out->threads = kThreads;
+    out->threads = uint32_t(ctx->threads_stats);
     out->chunk_elems = uint32_t(ctx->chunk_elems);
     out->launches = ctx->launches;
     out->misaligned_tensors = ctx->misaligned;
@@ -866,8 +991,8 @@ int static_setup(int dev, StaticSetup **out) {
         if (e != cudaSuccess)
             return fail(nullptr, GAC_ERR_CUDA, "cudaDeviceGetAttribute failed: %s (CUDA error %lld)",
                         cudaGetErrorString(e), (long long)e);
-        st.occ_f32 = resident_ctas(gac_stats_kernel<float>);
-        st.occ_bf16 = resident_ctas(gac_stats_kernel<bf16_t>);
+        st.occ_f32 = resident_ctas(gac_stats_kernel<float>, StatsGeom<float>::T);
+        st.occ_bf16 = resident_ctas(gac_stats_kernel<bf16_t>, StatsGeom<bf16_t>::T);
         st.base = static_cast<unsigned char *>(ptr);
         st.ready = true;
     }
@@ -943,10 +1068,10 @@ extern "C" int gac_stats_static(const gac_tensor *list, uint32_t n, int g_dtype,
     const int occ = g_dtype == GAC_BF16 ? st->occ_bf16 : st->occ_f32;
     const uint32_t grid = uint32_t(std::min<uint64_t>(std::min<uint64_t>(uint64_t(st->sms) * occ, kStaticMaxCtas), n_chunks));
     if (g_dtype == GAC_BF16)
-        gac_stats_kernel<bf16_t><<<grid, kThreads, 0, s>>>(d_chunks, uint32_t(n_chunks), d_partials, d_ticket,
+        gac_stats_kernel<bf16_t><<<grid, StatsGeom<bf16_t>::T, 0, s>>>(d_chunks, uint32_t(n_chunks), d_partials, d_ticket,
                                                            result_dev, nullptr, h);
     else
-        gac_stats_kernel<float><<<grid, kThreads, 0, s>>>(d_chunks, uint32_t(n_chunks), d_partials, d_ticket,
+        gac_stats_kernel<float><<<grid, StatsGeom<float>::T, 0, s>>>(d_chunks, uint32_t(n_chunks), d_partials, d_ticket,
                                                           result_dev, nullptr, h);
     GAC_CUDA(nullptr, cudaGetLastError());
     return GAC_OK;
