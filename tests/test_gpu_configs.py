@@ -1,0 +1,202 @@
+"""GPU parity on the benchmark configurations at their full sizes, in the
+launch configuration that bench.py times.
+
+The lists do not fit host memory as a whole (the 14 B list is 2 x 55 GiB), so
+the oracle is fed tensor by tensor: its three sums run over the whole list in
+list order; outputs are compared element by element on whole tensors up to
+32 M elements and on slices (head, an odd-offset middle, tail) of larger ones,
+after regenerating the pre-step values of that tensor from its seeds.  On top
+of that the state refresh d' = g is checked on every element of every tensor.
+"""
+import math
+import os
+
+import pytest
+import torch
+
+from oracle import gac_oracle as orc
+from paper_2603_01501_b200 import binding as gb
+from paper_2603_01501_b200 import synth
+
+from gpu_util import check_decision, check_sums, max_ulp, to_orc_hp
+
+pytestmark = pytest.mark.gpu
+
+THREADS = len(os.sched_getaffinity(0)) if hasattr(os, "sched_getaffinity") else 4
+FORCE = dict(c_low=0.05, c_high=2.0)
+FULL_LIMIT = 32 << 20
+SLICE = 4 << 20
+
+
+def oracle_sums_streamed(g_list, d_list, first_step=False):
+    big = max(t.numel() for t in g_list)
+    stage_g = torch.empty(big, dtype=g_list[0].dtype, pin_memory=True)
+    stage_d = torch.empty(big, dtype=torch.float32, pin_memory=True)
+    acc = orc.RunningStats(first_step=first_step, threads=THREADS)
+    for g, d in zip(g_list, d_list):
+        n = g.numel()
+        stage_g[:n].copy_(g)
+        stage_d[:n].copy_(d)
+        torch.cuda.synchronize()
+        acc.add(stage_g[:n], stage_d[:n])
+    return acc.value()
+
+
+def slices_of(n):
+    if n <= FULL_LIMIT:
+        return [(0, n)]
+    mid = (n // 2) | 1          # odd offset: not aligned to any vector or chunk boundary
+    return [(0, SLICE), (mid, mid + SLICE + 3), (n - SLICE - 1, n)]
+
+
+def check_outputs_sampled(shapes, rho, config_id, g_dtype, g_gpu, d_gpu, hp, dec):
+    ohp = to_orc_hp(hp)
+    lim = 4 if g_dtype == torch.float32 else 1
+    worst = 0
+    for i in range(len(shapes)):
+        (g0,), (d0,) = synth.gradient_list(shapes, rho, config_id, g_dtype, "cuda", indices=[i])
+        # state refresh: exact widening of the raw gradient, every element
+        assert torch.equal(d_gpu[i], g0.float()), f"tensor {i}: d' != raw g"
+        if dec.regime != orc.PROJECT:
+            assert torch.equal(g_gpu[i], g0), f"tensor {i}: g changed outside the projection regime"
+            continue
+        for lo, hi in slices_of(g0.numel()):
+            g_ref = g0[lo:hi].cpu().contiguous()
+            d_ref = d0[lo:hi].cpu().contiguous()
+            orc.project([g_ref], [d_ref], ohp, dec, threads=THREADS)
+            u = max_ulp(g_gpu[i][lo:hi].cpu(), g_ref)
+            assert u <= lim, f"tensor {i} [{lo}:{hi}]: g' differs by {u} ulp"
+            worst = max(worst, u)
+            assert torch.equal(d_gpu[i][lo:hi].cpu(), d_ref)
+        del g0, d0
+    return worst
+
+
+def run_config(workload, hp):
+    dims_key, g_dtype, rho, config_id = synth.WORKLOADS[workload]
+    shapes = synth.decoder_tensor_list(synth.DIMS[dims_key])
+    need = synth.list_numel(shapes) * ((2 if g_dtype == torch.bfloat16 else 4) + 4) + (12 << 30)
+    free, _ = torch.cuda.mem_get_info()
+    if free < need:
+        pytest.skip(f"needs {need >> 30} GiB of device memory, {free >> 30} GiB free")
+    g, d = synth.gradient_list(shapes, rho, config_id, g_dtype, "cuda")
+    dec = orc.decide(oracle_sums_streamed(g, d), to_orc_hp(hp))
+    ctx = gb.gac_init(g, d, hp)
+    res = gb.gac_stats(ctx, 2, staleness=1)
+    again = gb.gac_stats(ctx, 2, staleness=1)
+    assert (res.dot, res.gg, res.dd, res.cos) == (again.dot, again.gg, again.dd, again.cos)
+    check_sums(res, dec)
+    check_decision(res, dec)
+    assert abs(res.cos - rho) < 2e-3
+    gb.gac_project(ctx, coef_override=dec.coef if dec.regime == orc.PROJECT else None)
+    torch.cuda.synchronize()
+    worst = check_outputs_sampled(shapes, rho, config_id, g_dtype, g, d, hp, dec)
+    gb.gac_free(ctx)
+    del g, d
+    torch.cuda.empty_cache()
+    return res, dec, worst
+
+
+@pytest.mark.parametrize("workload", ["cfg2_1.5b_f32", "cfg3_7b_bf16", "cfg5_14b_f32"])
+def test_config_projection_regime(workload):
+    res, dec, worst = run_config(workload, gb.HParams(**FORCE))
+    assert res.regime == gb.GAC_REGIME_PROJECT
+    assert abs(res.alpha - 0.05 / abs(res.cos)) <= 1e-12
+
+
+@pytest.mark.parametrize("workload", ["cfg2_1.5b_f32", "cfg3_7b_bf16"])
+def test_config_paper_defaults_is_a_violation_step(workload):
+    # every configured cosine (0.8 .. 0.95) is above the paper's c_high = 0.3
+    res, dec, _ = run_config(workload, gb.HParams())
+    assert res.regime == gb.GAC_REGIME_VIOLATION
+
+
+# ------------------------------------------------------------ staleness runs
+
+def staleness_run(shapes, rho, k, run_id, steps, hp, full_outputs):
+    """Feeds the same exogenous gradient sequence to both sides, carrying the
+    stored direction across steps on each side independently."""
+    proc = synth.StalenessProcess(shapes, rho, k, config_id=4, run_id=run_id, device="cuda")
+    g = [torch.empty(n, device="cuda") for _, n in shapes]
+    d = [torch.full((n,), float("nan"), device="cuda") for _, n in shapes]
+    ctx = gb.gac_init(g, d, hp)
+    ohp = to_orc_hp(hp)
+    d_ref = [torch.full((n,), float("nan")) for _, n in shapes] if full_outputs else None
+    prev_raw = None
+    log = []
+    for t in range(1, steps + 1):
+        raw = proc.next()
+        for dst, src in zip(g, raw):
+            dst.copy_(src)
+        first = (t == 1)
+        if full_outputs:
+            g_ref = [x.cpu() for x in raw]
+            dec = orc.decide(orc.stats(g_ref, d_ref, first_step=first, threads=THREADS), ohp, first)
+            orc.project(g_ref, d_ref, ohp, dec, first_step=first, threads=THREADS)
+        else:
+            # the state is the previous raw gradient (checked bitwise below), so the oracle's
+            # sums for this step are those of (raw_t, raw_{t-1})
+            sums = oracle_sums_streamed(raw, prev_raw if prev_raw is not None else raw, first)
+            dec = orc.decide(sums, ohp, first)
+        res = gb.gac_stats(ctx, t, staleness=k)
+        gb.gac_project(ctx, coef_override=dec.coef if dec.regime == orc.PROJECT else None)
+        torch.cuda.synchronize()
+        check_sums(res, dec)
+        check_decision(res, dec)
+        for i, (a, b) in enumerate(zip(d, raw)):
+            assert torch.equal(a, b), f"step {t} tensor {i}: state is not the raw gradient"
+        if full_outputs:
+            lim = 4
+            for a, b in zip(g, g_ref):
+                assert max_ulp(a.cpu(), b) <= lim
+        elif dec.regime == orc.PROJECT:
+            # sampled outputs: one slice per tensor against the oracle
+            for i in range(0, len(shapes), 7):
+                n = shapes[i][1]
+                lo = (n // 3) | 1 if n > SLICE else 0
+                hi = min(n, lo + SLICE)
+                g_s = raw[i][lo:hi].cpu().contiguous()
+                d_s = prev_raw[i][lo:hi].cpu().contiguous()
+                orc.project([g_s], [d_s], ohp, dec)
+                assert max_ulp(g[i][lo:hi].cpu(), g_s) <= 4
+        prev_raw = raw
+        log.append((res.cos, res.regime, res.alpha))
+    gb.gac_free(ctx)
+    return log
+
+
+@pytest.mark.parametrize("rho", [0.0, 0.5, 0.95])
+@pytest.mark.parametrize("k", [1, 4, 8])
+def test_staleness_runs_scaled_down_all_steps(rho, k):
+    """64 consecutive steps for every (rho, k) on a scaled-down list of the same
+    structure, every element of every step compared."""
+    shapes = synth.decoder_tensor_list(synth.DIMS["mini"])
+    band = gb.HParams(c_low=0.05, c_high=0.99)
+    log = staleness_run(shapes, rho, k, run_id=int(rho * 100) * 10 + k, steps=64, hp=band,
+                        full_outputs=True)
+    assert log[0][1] == gb.GAC_REGIME_SAFE and log[0][0] == 0.0
+    cs = [abs(c) for c, _, _ in log[1 + k:]]
+    if rho == 0.0:
+        assert max(cs) < 0.05
+    else:
+        assert sum(cs) / len(cs) > 0.1
+    log2 = staleness_run(shapes, rho, k, run_id=int(rho * 100) * 10 + k, steps=12, hp=gb.HParams(),
+                         full_outputs=True)
+    assert [r for _, r, _ in log2][0] == gb.GAC_REGIME_SAFE
+
+
+def test_staleness_run_full_size_sample():
+    """The 1.5 B list at full size: a short run (the full 9 x 64 grid replayed by
+    the CPU oracle would take tens of minutes; set GAC_FULL_STALENESS=1 for it)."""
+    shapes = synth.decoder_tensor_list(synth.DIMS["1.5b"])
+    free, _ = torch.cuda.mem_get_info()
+    if free < (80 << 30):
+        pytest.skip("needs 80 GiB of device memory")
+    band = gb.HParams(c_low=0.05, c_high=0.99)
+    settings = [(0.5, 4, 6)]
+    if os.environ.get("GAC_FULL_STALENESS") == "1":
+        settings = [(r, k, 64) for r in (0.0, 0.5, 0.95) for k in (1, 4, 8)]
+    for rho, k, steps in settings:
+        log = staleness_run(shapes, rho, k, run_id=900 + k, steps=steps, hp=band, full_outputs=False)
+        assert log[0][1] == gb.GAC_REGIME_SAFE
+        assert any(r == gb.GAC_REGIME_PROJECT for _, r, _ in log[1:]) or rho == 0.0
