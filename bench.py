@@ -165,7 +165,7 @@ class Workload:
         if ev:
             ev[0].record()
         if self.world > 1:
-            # sharded form: local sums, ONE all-reduce of three numbers, same decision on every rank
+            # sharded form (App. A.1): local sums, ONE all-reduce of three numbers, same decision on every rank
             gb.gac_stats_partial(self.ctx, self.step_no, self.sums)
             torch.distributed.all_reduce(self.sums)
             gb.gac_decide(self.ctx, self.sums, fetch=False)

@@ -271,6 +271,34 @@ def test_sharded_partial_sums_add_up_to_the_whole():
         gb.gac_free(c)
 
 
+@pytest.mark.parametrize("world", [2, 3, 8])
+def test_flat_shard_plan_ranks_emulated_in_turn(world):
+    """FSDP-style flat shards (tensors cut at shard boundaries): the ranks' launches run one after
+    the other on this GPU, the sum of their three numbers stands for the all-reduce."""
+    from paper_2603_01501_b200 import sharding
+    shapes = synth.decoder_tensor_list(synth.DIMS["small"])
+    g, d = synth.gradient_list(shapes, 0.4, config_id=2, device="cuda")
+    hp = gb.HParams(**FORCE)
+    g_ref, d_ref = [t.cpu() for t in g], [t.cpu() for t in d]
+    dec = orc.decide(orc.stats(g_ref, d_ref), to_orc_hp(hp))
+    orc.project(g_ref, d_ref, to_orc_hp(hp), dec)
+    plan = sharding.flat_shard_plan([t.numel() for t in g], world)
+    ctxs = [gb.gac_init(sharding.shard_views(g, p), sharding.shard_views(d, p), hp) for p in plan]
+    bufs = [torch.zeros(3, dtype=torch.float64, device="cuda") for _ in plan]
+    for c, b in zip(ctxs, bufs):
+        gb.gac_stats_partial(c, 2, b)
+    total = torch.stack(bufs).sum(0)
+    for c in ctxs:
+        res = gb.gac_decide(c, total)
+        check_sums(res, dec)
+        check_decision(res, dec)
+        gb.gac_project(c, coef_override=dec.coef)
+    torch.cuda.synchronize()
+    check_outputs(g, d, g_ref, d_ref)
+    for c in ctxs:
+        gb.gac_free(c)
+
+
 def test_call_order_is_enforced():
     g, d = [torch.ones(100, device="cuda")], [torch.ones(100, device="cuda") * 2]
     ctx = gb.gac_init(g, d, gb.HParams())
