@@ -17,6 +17,7 @@ evicts the 126 MB L2.  Prints one JSON line.
 from __future__ import annotations
 
 import argparse
+import ctypes
 import hashlib
 import json
 import math
@@ -139,7 +140,7 @@ def recorded_traffic(kernel: str):
 # --------------------------------------------------------------- GPU workload
 
 class Workload:
-    def __init__(self, name: str, device, world: int):
+    def __init__(self, name: str, device, world: int, clip: float = 0.0):
         from paper_2603_01501_b200 import binding as gb
         self.gb = gb
         dims_key, self.g_dtype, self.rho, self.config_id = synth.WORKLOADS[name]
@@ -151,7 +152,7 @@ class Workload:
         self.scratch = torch.empty(max(n for _, n in self.shapes), dtype=torch.float32, device=device)
         self.gen = torch.Generator(device=device)
         self.gen.manual_seed(12345 + self.config_id)
-        self.ctx = gb.gac_init(self.g, self.d, gb.HParams(**FORCE))
+        self.ctx = gb.gac_init(self.g, self.d, gb.HParams(clip_max_norm=clip, **FORCE))
         self.step_no = 1      # the stored direction already holds g_{t-1}
         self.sums = torch.zeros(3, dtype=torch.float64, device=device) if world > 1 else None
 
@@ -206,6 +207,37 @@ def time_steps(wl: Workload, steps: int, warmup: int, sampler=None):
     return s_ms, p_ms
 
 
+def time_unchanged_regime(wl: Workload, steps: int):
+    """The same list under the paper's default thresholds (0.05, 0.3): every
+    configured cosine is above c_high, so these are violation steps -- the
+    reduction plus the state refresh d' = g with g left alone (a safe step moves
+    the same bytes)."""
+    gb = wl.gb
+    ctx = gb.gac_init(wl.g, wl.d, gb.HParams())
+    step_no = 1
+    evs = []
+    for i in range(3 + steps):
+        wl.refresh()
+        step_no += 1
+        e = [torch.cuda.Event(enable_timing=True) for _ in range(2)]
+        e[0].record()
+        gb.gac_stats(ctx, step_no, fetch=False)
+        gb.gac_project(ctx)
+        e[1].record()
+        if i >= 3:
+            evs.append(e)
+    res = gb.gac_stats(ctx, step_no + 1)
+    gb.gac_project(ctx)
+    torch.cuda.synchronize()
+    gb.gac_free(ctx)
+    ms = sum(a.elapsed_time(b) for a, b in evs) / len(evs)
+    sg = 2 if wl.g_dtype == torch.bfloat16 else 4
+    nbytes = wl.params * ((sg + 4) + sg + 4)
+    return {"regime": gb.REGIME_NAMES[res.regime], "ms_per_step": ms,
+            "value": wl.params / (ms * 1e-3), "unit": UNIT, "bytes_per_param": (sg + 4) + sg + 4,
+            "hbm_gbs": nbytes / (ms * 1e-3) / 1e9}
+
+
 class _Null:
     def __enter__(self):
         return self
@@ -244,7 +276,7 @@ def time_e2e(wl: Workload, steps: int, warmup: int):
         pinned = False
         host_g = [torch.empty(t.shape, dtype=t.dtype) for t in wl.g]
     h2d = sum(h.numel() * h.element_size() for h in host_g)
-    d2h = h2d + 72      # g' and the 72-byte decision record
+    d2h = h2d + ctypes.sizeof(gb.gac_result)      # g' and the decision record
     times = []
     for i in range(warmup + steps):
         wl.refresh()                       # next gradient, staged on the host (untimed)
@@ -386,6 +418,8 @@ def main():
     ap.add_argument("--workload", default="cfg3_7b_bf16", choices=sorted(synth.WORKLOADS))
     ap.add_argument("--also", default="cfg5_14b_f32",
                     help="second workload reported under 'also' (1 GPU only); 'none' to skip")
+    ap.add_argument("--clip", type=float, default=0.0,
+                    help="fold global-norm clipping with this max norm into the projection pass (0 = off)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
@@ -410,7 +444,7 @@ def main():
         torch.distributed.init_process_group("nccl", device_id=device)
     peak, peak_kind = measured_hbm_peak()
 
-    wl = Workload(args.workload, device, world)
+    wl = Workload(args.workload, device, world, args.clip)
     sampler = ClockSampler(nvml_index(local_rank))
     wall0 = time.perf_counter()
     s_ms, p_ms = time_steps(wl, args.steps, args.warmup, sampler)
@@ -431,7 +465,8 @@ def main():
             "hbm_gbs": summ["hbm_gbs"] , "frac_of_nominal_8TBs": summ["hbm_gbs"] / NOMINAL_HBM_GBS,
             "stats_ms": summ["stats_ms"], "project_ms": summ["project_ms"],
             "best_ms_per_step": summ["best_ms_per_step"],
-            "regime_check": {"cos": res.cos, "regime": gb.REGIME_NAMES[res.regime], "alpha": res.alpha},
+            "regime_check": {"cos": res.cos, "regime": gb.REGIME_NAMES[res.regime], "alpha": res.alpha,
+                             "clip_scale": res.clip_scale},
             "launch": {"grid": info.grid, "threads": info.threads, "chunk_elems": info.chunk_elems,
                        "chunks": info.n_chunks},
             "gpu_launches": (2 if world == 1 else 3) * args.steps,
@@ -441,6 +476,8 @@ def main():
         line["config"]["parallelism"] = (f"dp{world}: every rank holds one list as its gradient shard; "
                                          "one NCCL all-reduce of 3 doubles per step")
 
+    if world == 1:
+        line["unchanged_regime"] = time_unchanged_regime(wl, min(args.steps, 10))
     if not args.no_e2e:
         try:
             line["e2e"] = time_e2e(wl, min(args.steps, 5), 1)

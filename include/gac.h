@@ -59,7 +59,7 @@ typedef struct {
 } gac_tensor;
 
 /* Hyper-parameters.  Defaults of the paper: c_low 0.05, c_high 0.3 (App. C.3),
- * eps 1e-8 (App. A.1), beta 1 (App. A.2), adaptive mode, raw state. */
+ * eps 1e-8 (App. A.1), beta 1 (App. A.2), adaptive mode, raw state, no clipping. */
 typedef struct {
     double c_low, c_high;      /* Algorithm 1 inputs; ADAPTIVE mode needs 0 < c_low < c_high.
                                   c_high > 1 is legal and disables the skip branch.            */
@@ -73,6 +73,13 @@ typedef struct {
     int32_t zero_on_violation; /* 0: leave g alone, the caller skips its optimizer step
                                   (Algorithm 1: theta_t = theta_{t-1}); 1: write g' = 0          */
     int32_t reserved;          /* must be 0 */
+    double clip_max_norm;      /* > 0: global-norm clipping (Table 2 lists "Gradient clipping True")
+                                  folded into the projection pass: what a safe or projection step
+                                  sends on is scaled by min(1, clip_max_norm/(norm + clip_eps)),
+                                  with the norm taken in closed form from the three sums, so the
+                                  separate clipping pass of the optimizer is not needed.  0 = off.
+                                  The stored direction is never clipped.                           */
+    double clip_eps;           /* 1e-6 (the usual constant of global-norm clipping)                */
 } gac_hparams;
 
 /* What one step decided.  Lives on the device between gac_stats and
@@ -88,6 +95,10 @@ typedef struct {
     int32_t nonfinite;         /* 1 if a sum was NaN/Inf: regime = VIOLATION, g and d untouched  */
     uint32_t staleness;        /* echoed metadata: the rule never reads it                      */
     uint64_t step;             /* Algorithm 1's t for which this record holds                    */
+    double out_norm;           /* Euclidean norm of the gradient the step sends on, before clipping:
+                                  sqrt(beta^2 gg + 2 beta coef dot + coef^2 dd) when projecting, sqrt(gg)
+                                  when safe                                                       */
+    double clip_scale;         /* factor applied by clipping (1 when off, not needed, or skipped) */
 } gac_result;
 
 /* Fills *hp with the paper's defaults. */

@@ -195,6 +195,10 @@ typedef struct {
     double alpha_fixed;       /* parallel gain used when mode == FIXED              */
     int32_t zero_on_violation;
     int32_t reserved;
+    double clip_max_norm;     /* > 0: global-norm clipping of the outgoing gradient (Table 2:
+                                 "Gradient clipping True"), applied after the GAC rule; 0 = off */
+    double clip_eps;          /* added to the norm in the clip factor, 1e-6 as in torch's
+                                 clip_grad_norm_ */
 } orc_hparams;
 
 typedef struct {
@@ -263,11 +267,40 @@ void orc_decide(const double sums[3], const orc_hparams *hp, int first_step, orc
 
 /* ---- steps 5-6: in-place rank-one update and state refresh (App. A.2) ---- */
 
+/* Squared Euclidean norm of the gradient that the rule sends on, before any
+ * clipping and before rounding: sum over i of (beta g_i + coef d_i)^2 in the
+ * projection regime, of g_i^2 in the safe regime.  Accumulated into a->sum[0]
+ * with Neumaier compensation so that a list can be fed tensor by tensor. */
+void orc_outgoing_sqnorm(orc_acc *a, const void *g, int g_dt, const float *d, uint64_t n,
+                         const orc_hparams *hp, int regime, float coef, int d_is_zero)
+{
+    for (uint64_t i = 0; i < n; ++i) {
+        double gi = elem_as_double(g, g_dt, i);
+        double out = gi;
+        if (regime == ORC_PROJECT) {
+            double di = d_is_zero ? 0.0 : (double)d[i];
+            out = hp->beta * gi + (double)coef * di;
+        }
+        neumaier_add(&a->sum[0], &a->comp[0], out * out);
+    }
+}
+
+/* Global-norm clip factor: min(1, max_norm / (norm + clip_eps)). */
+double orc_clip_scale(double sqnorm, const orc_hparams *hp)
+{
+    if (!(hp->clip_max_norm > 0.0))
+        return 1.0;
+    double f = hp->clip_max_norm / (sqrt(sqnorm) + hp->clip_eps);
+    return f < 1.0 ? f : 1.0;
+}
+
 /* g (type g_dt) and d (binary32) are updated in place over n elements, given
  * the decision.  coef is the shared binary32 coefficient.  d_is_zero: d holds
- * no valid data on the first step and is only written. */
+ * no valid data on the first step and is only written.  clip_scale (1 = none)
+ * multiplies the outgoing gradient of a safe or projection step; a skipped
+ * step sends nothing on, so it is not scaled. */
 void orc_project(void *g, int g_dt, float *d, uint64_t n, const orc_hparams *hp, int regime,
-                 int nonfinite, float coef, int d_is_zero)
+                 int nonfinite, float coef, int d_is_zero, double clip_scale)
 {
     if (nonfinite)
         return;                        /* reading above: touch nothing */
@@ -281,6 +314,10 @@ void orc_project(void *g, int g_dt, float *d, uint64_t n, const orc_hparams *hp,
             write_g = 1;
         } else if (regime == ORC_VIOLATION && hp->zero_on_violation) {
             gout = 0.0;
+            write_g = 1;
+        }
+        if (clip_scale != 1.0 && regime != ORC_VIOLATION) {
+            gout = clip_scale * gout;
             write_g = 1;
         }
         if (write_g)

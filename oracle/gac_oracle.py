@@ -52,7 +52,8 @@ class _HParams(ctypes.Structure):
                 ("eps", ctypes.c_double), ("beta", ctypes.c_double),
                 ("mode", ctypes.c_int32), ("state_mode", ctypes.c_int32),
                 ("alpha_fixed", ctypes.c_double),
-                ("zero_on_violation", ctypes.c_int32), ("reserved", ctypes.c_int32)]
+                ("zero_on_violation", ctypes.c_int32), ("reserved", ctypes.c_int32),
+                ("clip_max_norm", ctypes.c_double), ("clip_eps", ctypes.c_double)]
 
 
 class _Decision(ctypes.Structure):
@@ -79,7 +80,12 @@ def lib():
         L.orc_decide.argtypes = [ctypes.c_double * 3, ctypes.POINTER(_HParams), i32,
                                  ctypes.POINTER(_Decision)]
         L.orc_project.argtypes = [vp, i32, vp, u64, ctypes.POINTER(_HParams), i32, i32,
-                                  ctypes.c_float, i32]
+                                  ctypes.c_float, i32, ctypes.c_double]
+        L.orc_outgoing_sqnorm.argtypes = [ctypes.POINTER(_Acc), vp, i32, vp, u64,
+                                          ctypes.POINTER(_HParams), i32, ctypes.c_float, i32]
+        L.orc_outgoing_sqnorm.restype = None
+        L.orc_clip_scale.argtypes = [ctypes.c_double, ctypes.POINTER(_HParams)]
+        L.orc_clip_scale.restype = ctypes.c_double
         L.orc_round_to_bf16.argtypes = [vp, vp, u64]
         for f in (L.orc_acc_init, L.orc_stats_accumulate, L.orc_acc_value, L.orc_acc_merge,
                   L.orc_stats_pairwise, L.orc_decide, L.orc_project, L.orc_round_to_bf16):
@@ -99,10 +105,13 @@ class HParams:
     alpha_fixed: float = 0.0
     state_mode: int = STATE_RAW
     zero_on_violation: int = 0
+    clip_max_norm: float = 0.0      # 0 = no clipping
+    clip_eps: float = 1e-6
 
     def c(self) -> _HParams:
         return _HParams(self.c_low, self.c_high, self.eps, self.beta, self.mode, self.state_mode,
-                        self.alpha_fixed, self.zero_on_violation, 0)
+                        self.alpha_fixed, self.zero_on_violation, 0, self.clip_max_norm,
+                        self.clip_eps)
 
 
 @dataclass
@@ -116,6 +125,8 @@ class Decision:
     coef: float          # binary32 value, held exactly in a Python float
     regime: int
     nonfinite: int
+    out_norm: float = float("nan")   # norm of the outgoing gradient before clipping (set by project)
+    clip_scale: float = 1.0          # factor applied by global-norm clipping (set by project)
 
 
 def _ptr_dt_n(t):
@@ -212,13 +223,39 @@ def decide(sums, hp: HParams, first_step: bool = False) -> Decision:
                     o.nonfinite)
 
 
-def project(g_list: Sequence, d_list: Sequence, hp: HParams, dec: Decision,
-            first_step: bool = False, coef: Optional[float] = None, threads: int = 1) -> None:
-    """In-place rank-one update of g and refresh of the stored direction d
-    (App. A.2).  `coef` overrides the decision's binary32 coefficient."""
+def outgoing_norm(g_list: Sequence, d_list: Sequence, hp: HParams, dec: Decision,
+                  first_step: bool = False, coef: Optional[float] = None) -> float:
+    """Euclidean norm of the (unrounded) gradient that a safe or projection step
+    sends on, by brute force over every element."""
     L = lib()
     chp = hp.c()
     k = dec.coef if coef is None else float(np.float32(coef))
+    acc = _Acc()
+    L.orc_acc_init(ctypes.byref(acc))
+    for g, d in zip(g_list, d_list):
+        gp, gdt, n = _ptr_dt_n(g)
+        dp, _, _ = _ptr_dt_n(d)
+        L.orc_outgoing_sqnorm(ctypes.byref(acc), gp, gdt, dp, n, ctypes.byref(chp), dec.regime,
+                              ctypes.c_float(k), 1 if first_step else 0)
+    out = (ctypes.c_double * 3)()
+    L.orc_acc_value(ctypes.byref(acc), out)
+    return float(out[0]) ** 0.5
+
+
+def project(g_list: Sequence, d_list: Sequence, hp: HParams, dec: Decision,
+            first_step: bool = False, coef: Optional[float] = None, threads: int = 1) -> None:
+    """In-place rank-one update of g and refresh of the stored direction d
+    (App. A.2), followed -- when hp.clip_max_norm > 0 -- by global-norm clipping
+    of what a safe or projection step sends on.  `coef` overrides the decision's
+    binary32 coefficient.  Records out_norm and clip_scale in `dec`."""
+    L = lib()
+    chp = hp.c()
+    k = dec.coef if coef is None else float(np.float32(coef))
+    scale = 1.0
+    if hp.clip_max_norm > 0 and not dec.nonfinite and dec.regime != VIOLATION:
+        dec.out_norm = outgoing_norm(g_list, d_list, hp, dec, first_step, coef)
+        scale = float(L.orc_clip_scale(dec.out_norm ** 2, ctypes.byref(chp)))
+    dec.clip_scale = scale
     jobs = []
     for g, d in zip(g_list, d_list):
         gp, gdt, n = _ptr_dt_n(g)
@@ -230,7 +267,8 @@ def project(g_list: Sequence, d_list: Sequence, hp: HParams, dec: Decision,
 
     def run(job):
         L.orc_project(job[0], job[1], job[2], job[3], ctypes.byref(chp), dec.regime,
-                      dec.nonfinite, ctypes.c_float(k), 1 if first_step else 0)
+                      dec.nonfinite, ctypes.c_float(k), 1 if first_step else 0,
+                      ctypes.c_double(scale))
 
     if threads <= 1:
         for job in jobs:

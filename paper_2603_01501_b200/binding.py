@@ -33,14 +33,16 @@ class gac_hparams(ctypes.Structure):
     _fields_ = [("c_low", ctypes.c_double), ("c_high", ctypes.c_double), ("eps", ctypes.c_double),
                 ("beta", ctypes.c_double), ("mode", ctypes.c_int32), ("state_mode", ctypes.c_int32),
                 ("alpha_fixed", ctypes.c_double), ("zero_on_violation", ctypes.c_int32),
-                ("reserved", ctypes.c_int32)]
+                ("reserved", ctypes.c_int32), ("clip_max_norm", ctypes.c_double),
+                ("clip_eps", ctypes.c_double)]
 
 
 class gac_result(ctypes.Structure):
     _fields_ = [("dot", ctypes.c_double), ("gg", ctypes.c_double), ("dd", ctypes.c_double),
                 ("cos", ctypes.c_double), ("alpha", ctypes.c_double), ("coef64", ctypes.c_double),
                 ("coef", ctypes.c_float), ("regime", ctypes.c_int32), ("nonfinite", ctypes.c_int32),
-                ("staleness", ctypes.c_uint32), ("step", ctypes.c_uint64)]
+                ("staleness", ctypes.c_uint32), ("step", ctypes.c_uint64),
+                ("out_norm", ctypes.c_double), ("clip_scale", ctypes.c_double)]
 
     def as_dict(self):
         return {k: getattr(self, k) for k, _ in self._fields_}
@@ -113,10 +115,13 @@ class HParams:
     alpha_fixed: float = 0.0
     state_mode: int = GAC_STATE_RAW
     zero_on_violation: int = 0
+    clip_max_norm: float = 0.0     # > 0 folds global-norm clipping into the projection pass
+    clip_eps: float = 1e-6
 
     def c(self) -> gac_hparams:
         return gac_hparams(self.c_low, self.c_high, self.eps, self.beta, self.mode,
-                           self.state_mode, self.alpha_fixed, self.zero_on_violation, 0)
+                           self.state_mode, self.alpha_fixed, self.zero_on_violation, 0,
+                           self.clip_max_norm, self.clip_eps)
 
 
 _DT = {torch.float32: GAC_F32, torch.bfloat16: GAC_BF16}
@@ -248,7 +253,7 @@ def gac_stats_static(g_list: Sequence[torch.Tensor], d_list: Sequence[torch.Tens
     L = load_library()
     if not (result_dev.is_cuda and result_dev.dtype == torch.uint8 and result_dev.is_contiguous()
             and result_dev.numel() >= ctypes.sizeof(gac_result) and result_dev.data_ptr() % 8 == 0):
-        raise ValueError("result_dev must be an 8-byte aligned CUDA uint8 tensor of >= 72 bytes")
+        raise ValueError("result_dev must be an 8-byte aligned CUDA uint8 tensor of >= sizeof(gac_result) bytes")
     n = len(g_list)
     arr = (gac_tensor * max(n, 1))()
     for i, (g, d) in enumerate(zip(g_list, d_list)):

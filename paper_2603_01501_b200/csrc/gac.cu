@@ -120,6 +120,7 @@ struct DevHP {
     unsigned long long step;
     unsigned staleness;
     int decide;      // 0: only publish the three sums (sharded form)
+    double clip_max, clip_eps;
 };
 
 struct F4 {
@@ -232,6 +233,26 @@ __device__ __forceinline__ Chunk load_chunk(const Chunk *table, uint32_t c) {
 
 // ------------------------------------------------------- decision (O(1) work)
 
+// Global-norm clipping folded into the update (Table 2: "Gradient clipping
+// True").  The squared norm of what a step sends on follows from the three
+// sums alone: |beta g + k d|^2 = beta^2 <g,g> + 2 beta k <g,d> + k^2 <d,d> in the
+// projection regime (k = the binary32 coefficient actually applied), <g,g> in
+// the safe regime; a skipped step sends nothing on.  Factor as in the usual
+// global-norm clip: min(1, max_norm / (norm + clip_eps)).
+__device__ __forceinline__ double clip_factor(int regime, double dot, double gg, double dd, double beta,
+                                              double k, double clip_max, double clip_eps, double *norm_out) {
+    double n2 = gg;
+    if (regime == GAC_REGIME_PROJECT)
+        n2 = __dadd_rn(__dadd_rn(__dmul_rn(__dmul_rn(beta, beta), gg),
+                                 __dmul_rn(__dmul_rn(2.0 * beta, k), dot)),
+                       __dmul_rn(__dmul_rn(k, k), dd));
+    const double norm = __dsqrt_rn(fmax(n2, 0.0));
+    *norm_out = norm;
+    if (!(clip_max > 0.0) || regime == GAC_REGIME_VIOLATION) return 1.0;
+    const double f = __ddiv_rn(clip_max, __dadd_rn(norm, clip_eps));
+    return f < 1.0 ? f : 1.0;
+}
+
 // Cosine with eps outside the root (App. A.1), the inclusive branches of
 // Algorithm 1, alpha = c_low/|c| (Eq. 5) or the caller's gain (Eq. 3), and the
 // multiplier of d in the rank-one form of App. A.2.
@@ -246,6 +267,8 @@ __device__ void take_decision(double dot, double gg, double dd, const DevHP &hp,
     r->alpha = 1.0;
     r->coef64 = 0.0;
     r->coef = 0.0f;
+    r->out_norm = 0.0;
+    r->clip_scale = 1.0;
     r->staleness = hp.staleness;
     r->step = hp.step;
     r->nonfinite = !(isfinite(dot) && isfinite(gg) && isfinite(dd));
@@ -257,6 +280,7 @@ __device__ void take_decision(double dot, double gg, double dd, const DevHP &hp,
     if (gg == 0.0 || dd == 0.0) {   // zero reference: u = 0, projector = identity
         r->cos = 0.0;
         r->regime = GAC_REGIME_SAFE;
+        r->clip_scale = clip_factor(r->regime, dot, gg, dd, hp.beta, 0.0, hp.clip_max, hp.clip_eps, &r->out_norm);
         return;
     }
     double c = __ddiv_rn(dot, __dadd_rn(__dsqrt_rn(__dmul_rn(gg, dd)), hp.eps));
@@ -267,6 +291,7 @@ __device__ void take_decision(double dot, double gg, double dd, const DevHP &hp,
         r->alpha = hp.alpha_fixed;
     } else if (ac <= hp.c_low) {
         r->regime = GAC_REGIME_SAFE;
+        r->clip_scale = clip_factor(r->regime, dot, gg, dd, hp.beta, 0.0, hp.clip_max, hp.clip_eps, &r->out_norm);
         return;
     } else if (ac >= hp.c_high) {
         r->regime = GAC_REGIME_VIOLATION;
@@ -278,6 +303,8 @@ __device__ void take_decision(double dot, double gg, double dd, const DevHP &hp,
     double k = __ddiv_rn(__dmul_rn(__dadd_rn(r->alpha, -hp.beta), dot), dd);
     r->coef64 = k;
     r->coef = __double2float_rn(k);
+    r->clip_scale = clip_factor(r->regime, dot, gg, dd, hp.beta, double(r->coef), hp.clip_max, hp.clip_eps,
+                                &r->out_norm);
 }
 
 // ------------------------------------------------------------- stats kernel
@@ -434,23 +461,25 @@ __global__ void gac_decide_kernel(const double *sums_in, gac_result *rec, DevHP 
 
 // ----------------------------------------------------------- project kernel
 
-enum GOp { G_KEEP = 0, G_FMA = 1, G_ZERO = 2 };
+enum GOp { G_KEEP = 0, G_FMA = 1, G_ZERO = 2, G_SCALE = 3 };
 enum DOp { D_KEEP = 0, D_RAW = 1, D_NEW = 2 };
 
 template <bool BETA1>
-__device__ __forceinline__ float rank_one(float g, float d, float k, double beta) {
-    if (BETA1) return fmaf(k, d, g);   // one rounding
-    // general beta: the sum of a rounded product and an exact product, in binary64
-    return __double2float_rn(__dadd_rn(__dmul_rn(beta, double(g)), __dmul_rn(double(k), double(d))));
+__device__ __forceinline__ float rank_one(float g, float d, float k, double beta, double s) {
+    if (BETA1) return fmaf(k, d, g);   // beta = 1, no clipping: one rounding
+    // general beta and/or an active clip factor s: binary64 (rounded product + exact product), times s
+    return __double2float_rn(
+        __dmul_rn(s, __dadd_rn(__dmul_rn(beta, double(g)), __dmul_rn(double(k), double(d)))));
 }
+__device__ __forceinline__ float scaled(float g, double s) { return __double2float_rn(__dmul_rn(s, double(g))); }
 
 template <typename GT, int GOP, int DOP, bool BETA1>
-__device__ __forceinline__ void project_chunk(const Chunk &ch, float k, double beta) {
+__device__ __forceinline__ void project_chunk(const Chunk &ch, float k, double beta, double s) {
     void *g = reinterpret_cast<void *>(ch.g);
     void *d = reinterpret_cast<void *>(ch.d);
     const uint32_t tid = threadIdx.x;
     constexpr int T = ProjGeom<GT>::T, U = ProjGeom<GT>::U;
-    constexpr bool kReadG = (GOP == G_FMA) || (DOP == D_RAW);
+    constexpr bool kReadG = (GOP == G_FMA) || (GOP == G_SCALE) || (DOP == D_RAW);
     constexpr bool kReadD = (GOP == G_FMA);
     if (ch.flags & kChunkAligned) {
         const uint32_t nvec = ch.n >> 2;
@@ -473,15 +502,16 @@ __device__ __forceinline__ void project_chunk(const Chunk &ch, float k, double b
                 F4 out = gv[u];
                 if (GOP == G_ZERO) out = F4{0.f, 0.f, 0.f, 0.f};
                 if (GOP == G_FMA) {
-                    out.x = rank_one<BETA1>(gv[u].x, dv[u].x, k, beta);
-                    out.y = rank_one<BETA1>(gv[u].y, dv[u].y, k, beta);
-                    out.z = rank_one<BETA1>(gv[u].z, dv[u].z, k, beta);
-                    out.w = rank_one<BETA1>(gv[u].w, dv[u].w, k, beta);
+                    out.x = rank_one<BETA1>(gv[u].x, dv[u].x, k, beta, s);
+                    out.y = rank_one<BETA1>(gv[u].y, dv[u].y, k, beta, s);
+                    out.z = rank_one<BETA1>(gv[u].z, dv[u].z, k, beta, s);
+                    out.w = rank_one<BETA1>(gv[u].w, dv[u].w, k, beta, s);
                 }
+                if (GOP == G_SCALE) out = F4{scaled(gv[u].x, s), scaled(gv[u].y, s), scaled(gv[u].z, s), scaled(gv[u].w, s)};
                 if (GOP != G_KEEP) Elem<GT>::store4(g, v, out);
                 if (DOP == D_RAW) Elem<float>::store4(d, v, gv[u]);
                 if (DOP == D_NEW) {
-                    if (GOP == G_FMA) out = Elem<GT>::template load4<GAC_LD_PROJECT>(g, v);   // the value as stored (rounded)
+                    if (GOP == G_FMA || GOP == G_SCALE) out = Elem<GT>::template load4<GAC_LD_PROJECT>(g, v);   // the value as stored (rounded)
                     Elem<float>::store4(d, v, out);
                 }
             }
@@ -491,11 +521,12 @@ __device__ __forceinline__ void project_chunk(const Chunk &ch, float k, double b
             const uint32_t i = done + tid;
             const float x = kReadG ? Elem<GT>::load1(g, i) : 0.f;
             float out = (GOP == G_ZERO) ? 0.f : x;
-            if (GOP == G_FMA) out = rank_one<BETA1>(x, Elem<float>::load1(d, i), k, beta);
+            if (GOP == G_FMA) out = rank_one<BETA1>(x, Elem<float>::load1(d, i), k, beta, s);
+            if (GOP == G_SCALE) out = scaled(x, s);
             if (GOP != G_KEEP) Elem<GT>::store1(g, i, out);
             if (DOP == D_RAW) Elem<float>::store1(d, i, x);
             if (DOP == D_NEW) {
-                if (GOP == G_FMA) out = Elem<GT>::load1(g, i);
+                if (GOP == G_FMA || GOP == G_SCALE) out = Elem<GT>::load1(g, i);
                 Elem<float>::store1(d, i, out);
             }
         }
@@ -503,11 +534,12 @@ __device__ __forceinline__ void project_chunk(const Chunk &ch, float k, double b
         for (uint32_t i = tid; i < ch.n; i += T) {
             const float x = kReadG ? Elem<GT>::load1(g, i) : 0.f;
             float out = (GOP == G_ZERO) ? 0.f : x;
-            if (GOP == G_FMA) out = rank_one<BETA1>(x, Elem<float>::load1(d, i), k, beta);
+            if (GOP == G_FMA) out = rank_one<BETA1>(x, Elem<float>::load1(d, i), k, beta, s);
+            if (GOP == G_SCALE) out = scaled(x, s);
             if (GOP != G_KEEP) Elem<GT>::store1(g, i, out);
             if (DOP == D_RAW) Elem<float>::store1(d, i, x);
             if (DOP == D_NEW) {
-                if (GOP == G_FMA) out = Elem<GT>::load1(g, i);
+                if (GOP == G_FMA || GOP == G_SCALE) out = Elem<GT>::load1(g, i);
                 Elem<float>::store1(d, i, out);
             }
         }
@@ -516,9 +548,9 @@ __device__ __forceinline__ void project_chunk(const Chunk &ch, float k, double b
 
 template <typename GT, int GOP, int DOP, bool BETA1>
 __device__ __forceinline__ void project_walk(const Chunk *chunks, uint32_t n_chunks, float k,
-                                             double beta) {
+                                             double beta, double s) {
     for (uint32_t c = blockIdx.x; c < n_chunks; c += gridDim.x)
-        project_chunk<GT, GOP, DOP, BETA1>(load_chunk(chunks, c), k, beta);
+        project_chunk<GT, GOP, DOP, BETA1>(load_chunk(chunks, c), k, beta, s);
 }
 
 // The regime is read from the device-resident record, so no host round trip
@@ -527,22 +559,35 @@ __device__ __forceinline__ void project_walk(const Chunk *chunks, uint32_t n_chu
 // compile time so that each instantiation holds only the loops it can reach.
 template <typename GT, int STATE, bool BETA1, bool ZERO>
 __global__ void __launch_bounds__(ProjGeom<GT>::T, ProjGeom<GT>::MINB)
-gac_project_kernel(const Chunk *__restrict__ chunks, uint32_t n_chunks, const gac_result *rec,
-                   float coef_override, int use_override, double beta) {
+gac_project_kernel(const Chunk *__restrict__ chunks, uint32_t n_chunks, gac_result *rec,
+                   float coef_override, int use_override, double beta, double clip_max, double clip_eps) {
     if (rec->nonfinite) return;   // reading taken for NaN/Inf: touch nothing
     const int regime = rec->regime;
     const float k = use_override ? coef_override : rec->coef;
     constexpr int dop = STATE == GAC_STATE_RAW ? D_RAW : (STATE == GAC_STATE_PROJECTED ? D_NEW : D_KEEP);
+    double s = 1.0;
+    if (clip_max > 0.0) {
+        // recomputed here so that it belongs to the coefficient actually applied
+        double norm;
+        s = clip_factor(regime, rec->dot, rec->gg, rec->dd, beta, double(k), clip_max, clip_eps, &norm);
+        if (use_override && blockIdx.x == 0 && threadIdx.x == 0) {
+            rec->out_norm = norm;       // nobody reads these two fields during this launch
+            rec->clip_scale = s;
+        }
+    }
     if (regime == GAC_REGIME_PROJECT) {
-        project_walk<GT, G_FMA, dop, BETA1>(chunks, n_chunks, k, beta);
+        if (s != 1.0) project_walk<GT, G_FMA, dop, false>(chunks, n_chunks, k, beta, s);
+        else project_walk<GT, G_FMA, dop, BETA1>(chunks, n_chunks, k, beta, 1.0);
     } else if (ZERO && regime == GAC_REGIME_VIOLATION) {
-        project_walk<GT, G_ZERO, dop, true>(chunks, n_chunks, k, 1.0);
+        project_walk<GT, G_ZERO, dop, true>(chunks, n_chunks, k, 1.0, 1.0);
+    } else if (s != 1.0) {
+        project_walk<GT, G_SCALE, dop, true>(chunks, n_chunks, k, 1.0, s);   // safe step, clipped: g'' = s g
     } else if (STATE != GAC_STATE_HOLD) {
-        project_walk<GT, G_KEEP, D_RAW, true>(chunks, n_chunks, k, 1.0);   // d' = g, g untouched
+        project_walk<GT, G_KEEP, D_RAW, true>(chunks, n_chunks, k, 1.0, 1.0);   // d' = g, g untouched
     }
 }
 
-using ProjectKernel = void (*)(const Chunk *, uint32_t, const gac_result *, float, int, double);
+using ProjectKernel = void (*)(const Chunk *, uint32_t, gac_result *, float, int, double, double, double);
 
 template <typename GT, int STATE>
 ProjectKernel pick_project(bool beta1, bool zero) {
@@ -720,6 +765,8 @@ int check_hparams(const gac_hparams *hp) {
     if (hp->zero_on_violation != 0 && hp->zero_on_violation != 1)
         return fail(nullptr, GAC_ERR_INVALID_ARG, "zero_on_violation must be 0 or 1%s");
     if (hp->reserved != 0) return fail(nullptr, GAC_ERR_INVALID_ARG, "reserved field must be 0%s");
+    if (!(hp->clip_max_norm >= 0.0) || !isfinite(hp->clip_max_norm) || !(hp->clip_eps >= 0.0) || !isfinite(hp->clip_eps))
+        return fail(nullptr, GAC_ERR_INVALID_ARG, "clip_max_norm and clip_eps must be finite and >= 0%s");
     return GAC_OK;
 }
 
@@ -737,6 +784,8 @@ DevHP dev_hp(const gac_ctx *c, uint64_t step, uint32_t staleness, int decide) {
     h.step = step;
     h.staleness = staleness;
     h.decide = decide;
+    h.clip_max = c->hp.clip_max_norm;
+    h.clip_eps = c->hp.clip_eps;
     return h;
 }
 
@@ -781,6 +830,8 @@ void gac_default_hparams(gac_hparams *hp) {
     hp->beta = 1.0;
     hp->mode = GAC_MODE_ADAPTIVE;
     hp->state_mode = GAC_STATE_RAW;
+    hp->clip_max_norm = 0.0;
+    hp->clip_eps = 1e-6;
 }
 
 int gac_init(gac_ctx **out, const gac_tensor *list, uint32_t n, int g_dtype, int d_dtype,
@@ -911,7 +962,7 @@ int gac_project(gac_ctx *ctx, void *cuda_stream, const float *coef_override, gac
     const int use = coef_override ? 1 : 0;
     const uint32_t nc = uint32_t(ctx->n_chunks);
     reinterpret_cast<ProjectKernel>(const_cast<void *>(ctx->project_fn))<<<ctx->grid_project, ctx->threads_project, 0, s>>>(
-        ctx->d_chunks, nc, ctx->d_rec, k, use, ctx->hp.beta);
+        ctx->d_chunks, nc, ctx->d_rec, k, use, ctx->hp.beta, ctx->hp.clip_max_norm, ctx->hp.clip_eps);
     GAC_CUDA(ctx, cudaGetLastError());
     ++ctx->launches;
     ctx->decision_ready = false;

@@ -24,7 +24,8 @@ REL = 1e-5
 def to_orc_hp(hp: gb.HParams) -> orc.HParams:
     return orc.HParams(c_low=hp.c_low, c_high=hp.c_high, eps=hp.eps, beta=hp.beta, mode=hp.mode,
                        alpha_fixed=hp.alpha_fixed, state_mode=hp.state_mode,
-                       zero_on_violation=hp.zero_on_violation)
+                       zero_on_violation=hp.zero_on_violation, clip_max_norm=hp.clip_max_norm,
+                       clip_eps=hp.clip_eps)
 
 
 def ordered_int(t: torch.Tensor) -> torch.Tensor:
@@ -98,7 +99,9 @@ def step_both(g_cpu, d_cpu, hp: gb.HParams, step=2, device="cuda", launch=None, 
     if launch:
         gb.gac_set_launch(ctx, *launch)
     res = gb.gac_stats(ctx, step)
-    gb.gac_project(ctx, coef_override=dec.coef if (same_coef and dec.regime == orc.PROJECT) else None)
+    after = gb.gac_project(ctx, coef_override=dec.coef if (same_coef and dec.regime == orc.PROJECT) else None,
+                           fetch=True)
     torch.cuda.synchronize()
     gb.gac_free(ctx)
+    res.after = after            # the record as it stands after the projection pass
     return res, dec, g_gpu, d_gpu, g_ref, d_ref

@@ -175,6 +175,28 @@ def test_variants(hp, g_dtype):
     check_outputs(gg, dg, gr, dr, d_follows_g=follows)
 
 
+@pytest.mark.parametrize("g_dtype", [torch.float32, torch.bfloat16], ids=["f32", "bf16"])
+@pytest.mark.parametrize("max_norm", [1e-3, 0.3, 1e6])
+@pytest.mark.parametrize("thr", [FORCE, dict(c_low=0.9, c_high=0.95), dict()], ids=["project", "safe", "violation"])
+def test_clipping_folded_into_the_projection_pass(thr, max_norm, g_dtype):
+    """Global-norm clipping (Table 2) from the closed-form norm: same factor and
+    same outputs as the oracle's brute-force norm over every element."""
+    shapes = synth.decoder_tensor_list(synth.DIMS["small"])
+    g, d = synth.gradient_list(shapes, 0.6, config_id=2, g_dtype=g_dtype)
+    hp = gb.HParams(clip_max_norm=max_norm, **thr)
+    res, dec, gg, dg, gr, dr = step_both(g, d, hp)
+    check_sums(res, dec)
+    check_decision(res, dec)
+    after = res.after
+    if dec.regime == orc.VIOLATION:
+        assert after.clip_scale == 1.0 and dec.clip_scale == 1.0
+    else:
+        assert abs(after.out_norm - dec.out_norm) <= 1e-9 * dec.out_norm
+        assert abs(after.clip_scale - dec.clip_scale) <= 1e-9 * dec.clip_scale
+        assert (dec.clip_scale < 1.0) == (max_norm < 1e6)
+    check_outputs(gg, dg, gr, dr)
+
+
 def test_degenerate_vectors():
     n = 5000
     g, d = rand_pair(n, 0.5, seed=9)

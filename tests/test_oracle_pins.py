@@ -372,3 +372,63 @@ def test_bf16_gradient_list_path():
     x = g0.double().numpy() + dec.coef * d0.double().numpy()
     ulp = 2.0 ** (np.floor(np.log2(np.abs(x))) - 7)
     assert np.all(np.abs(g.double().numpy() - x) <= 0.5 * ulp * (1 + 1e-12))
+
+
+# ------------------------------------------------- global-norm clipping (Table 2)
+
+def test_clipping_matches_library_clip_after_the_rule():
+    """Clipping folded into the update must equal the unclipped rule followed by the
+    library's global-norm clip (torch.nn.utils.clip_grad_norm_), up to the extra
+    rounding the two-pass form makes."""
+    shapes = synth.decoder_tensor_list(synth.DIMS["mini"])
+    gl, dl = synth.gradient_list(shapes, 0.2, 2)
+    for max_norm in (1e-3, 0.05, 1e6):
+        hp0 = orc.HParams(c_low=0.05, c_high=0.9)
+        hp1 = orc.HParams(c_low=0.05, c_high=0.9, clip_max_norm=max_norm)
+        g0, d0 = [t.clone() for t in gl], [t.clone() for t in dl]
+        g1, d1 = [t.clone() for t in gl], [t.clone() for t in dl]
+        dec0 = orc.step(g0, d0, hp0)
+        dec1 = orc.step(g1, d1, hp1)
+        assert dec0.regime == dec1.regime == orc.PROJECT
+        params = [torch.nn.Parameter(torch.zeros_like(t)) for t in g0]
+        for p_, t in zip(params, g0):
+            p_.grad = t.clone()
+        total = float(torch.nn.utils.clip_grad_norm_(params, max_norm))
+        assert dec1.out_norm == pytest.approx(total, rel=1e-6)
+        if max_norm == 1e6:
+            assert dec1.clip_scale == 1.0
+            for a, b in zip(g1, g0):
+                np.testing.assert_array_equal(a.numpy(), b.numpy())
+        else:
+            assert dec1.clip_scale == pytest.approx(max_norm / (total + 1e-6), rel=1e-6)
+            for a, p_ in zip(g1, params):
+                # the library rounds g', the factor and the product to binary32: a few ulp apart
+                np.testing.assert_allclose(a.numpy(), p_.grad.numpy(), rtol=5e-7, atol=0)
+        for a, b in zip(d1, d0):
+            np.testing.assert_array_equal(a.numpy(), b.numpy())      # the state is never clipped
+
+
+def test_clipping_closed_forms_and_regimes():
+    g, d = synth.flat_pair_with_cosine(1 << 12, 0.6, s=2.0, seed=12)
+    g, d = g.numpy(), d.numpy()
+    hp = orc.HParams(c_low=0.05, c_high=0.95, eps=0.0, clip_max_norm=0.5)
+    g1, d1 = g.copy(), d.copy()
+    dec = orc.step([g1], [d1], hp)
+    c, cl = dec.cos, hp.c_low
+    assert dec.out_norm ** 2 == pytest.approx(dec.gg * (1 - c * c + cl * cl), rel=1e-6)
+    assert dec.clip_scale == pytest.approx(0.5 / (dec.out_norm + 1e-6), rel=1e-12)
+    assert math.sqrt(dot64(g1, g1)) == pytest.approx(0.5 * dec.out_norm / (dec.out_norm + 1e-6),
+                                                     rel=1e-6)
+    # safe step: only the clip acts, g'' = s g
+    w = np.random.default_rng(0).standard_normal(g.size).astype(np.float32)
+    w -= np.float32(dot64(w, d) / dot64(d, d)) * d
+    g2, d2 = w.copy(), d.copy()
+    dec = orc.step([g2], [d2], orc.HParams(clip_max_norm=1.0))
+    assert dec.regime == orc.SAFE and dec.clip_scale < 1.0
+    np.testing.assert_allclose(g2, w.astype(np.float64) * dec.clip_scale, rtol=6e-8)
+    np.testing.assert_array_equal(d2, w)
+    # skipped step: nothing is sent on, nothing is scaled
+    g3, d3 = (d * 3).astype(np.float32), d.copy()
+    dec = orc.step([g3], [d3], orc.HParams(clip_max_norm=1e-3))
+    assert dec.regime == orc.VIOLATION and dec.clip_scale == 1.0
+    np.testing.assert_array_equal(g3, (d * 3).astype(np.float32))
