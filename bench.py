@@ -238,6 +238,50 @@ def time_unchanged_regime(wl: Workload, steps: int):
             "hbm_gbs": nbytes / (ms * 1e-3) / 1e9}
 
 
+def time_fused_adamw(wl: Workload, steps: int):
+    """stats + the projection fused with AdamW (Table 2 values): the update goes
+    straight into p, m, v and g' is never written.  Moves (sg+4) + (sg+4+12) read
+    + 16 written bytes per parameter."""
+    gb = wl.gb
+    free, _ = torch.cuda.mem_get_info()
+    need = wl.params * 12 + (2 << 30)
+    if free < need:
+        return {"skipped": f"needs {need} bytes of device memory for p, m, v; {free} free"}
+    p = [torch.randn(t.numel(), device=wl.device) * 0.02 for t in wl.g]
+    m = [torch.zeros(t.numel(), device=wl.device) for t in wl.g]
+    v = [torch.zeros(t.numel(), device=wl.device) for t in wl.g]
+    ctx = gb.gac_init(wl.g, wl.d, gb.HParams(**FORCE))
+    gb.gac_attach_adamw(ctx, p, m, v, 0)
+    opt = gb.AdamW()
+    step_no, evs = 1, []
+    for i in range(3 + steps):
+        wl.refresh()
+        step_no += 1
+        e = [torch.cuda.Event(enable_timing=True) for _ in range(3)]
+        e[0].record()
+        gb.gac_stats(ctx, step_no, fetch=False)
+        e[1].record()
+        gb.gac_project_adamw(ctx, opt)
+        e[2].record()
+        if i >= 3:
+            evs.append(e)
+    torch.cuda.synchronize()
+    gb.gac_stats(ctx, step_no + 1, fetch=False)
+    res = gb.gac_project_adamw(ctx, opt, fetch=True)
+    gb.gac_free(ctx)
+    s_ms = sum(a.elapsed_time(b) for a, b, _ in evs) / len(evs)
+    f_ms = sum(b.elapsed_time(c) for _, b, c in evs) / len(evs)
+    sg = 2 if wl.g_dtype == torch.bfloat16 else 4
+    fused_bytes = wl.params * ((sg + 4 + 12) + 16)
+    del p, m, v
+    torch.cuda.empty_cache()
+    return {"ms_per_step": s_ms + f_ms, "stats_ms": s_ms, "fused_ms": f_ms,
+            "value": wl.params / ((s_ms + f_ms) * 1e-3), "unit": UNIT,
+            "fused_bytes_per_param": (sg + 4 + 12) + 16,
+            "fused_kernel_gbs": fused_bytes / (f_ms * 1e-3) / 1e9,
+            "applied_steps": res.applied_steps, "regime": gb.REGIME_NAMES[res.regime]}
+
+
 class _Null:
     def __enter__(self):
         return self
@@ -420,6 +464,8 @@ def main():
                     help="second workload reported under 'also' (1 GPU only); 'none' to skip")
     ap.add_argument("--clip", type=float, default=0.0,
                     help="fold global-norm clipping with this max norm into the projection pass (0 = off)")
+    ap.add_argument("--adamw", action="store_true",
+                    help="also time the projection fused with AdamW on the main workload (1 GPU)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
@@ -478,6 +524,8 @@ def main():
 
     if world == 1:
         line["unchanged_regime"] = time_unchanged_regime(wl, min(args.steps, 10))
+    if world == 1 and args.adamw:
+        line["fused_adamw"] = time_fused_adamw(wl, min(args.steps, 10))
     if not args.no_e2e:
         try:
             line["e2e"] = time_e2e(wl, min(args.steps, 5), 1)

@@ -99,6 +99,8 @@ typedef struct {
                                   sqrt(beta^2 gg + 2 beta coef dot + coef^2 dd) when projecting, sqrt(gg)
                                   when safe                                                       */
     double clip_scale;         /* factor applied by clipping (1 when off, not needed, or skipped) */
+    uint64_t applied_steps;    /* optimizer updates applied so far by gac_project_adamw (skipped steps
+                                  do not count); kept on the device across steps                  */
 } gac_result;
 
 /* Fills *hp with the paper's defaults. */
@@ -175,6 +177,41 @@ int gac_decide(gac_ctx *ctx, void *cuda_stream, const double *sums_in, gac_resul
  *   host_out         as in gac_stats
  */
 int gac_project(gac_ctx *ctx, void *cuda_stream, const float *coef_override, gac_result *host_out);
+
+/*
+ * The step after the path: the update handed straight to the optimizer.
+ * Algorithm 1 ends each safe or projection step with theta_t = theta_{t-1} +
+ * eta g' and the paper trains with AdamW (Table 2: lr 1e-6, betas (0.9, 0.999),
+ * eps 1e-8, weight decay 1e-2, gradient clipping on).  gac_project_adamw is
+ * gac_project and that optimizer step in ONE pass: it reads g, d, p, m, v once,
+ * writes d' = g and the new p, m, v, and never writes g' back (g is left as it
+ * was), which saves the separate optimizer pass over g'.
+ *     g' = clip_scale (beta g + coef d)   (projection)   or  clip_scale g   (safe)
+ *     p <- p (1 - lr wd);  m <- b1 m + (1-b1) g';  v <- b2 v + (1-b2) g'^2
+ *     p <- p - lr/(1-b1^t) * m / (sqrt(v)/sqrt(1-b2^t) + eps),  t = applied_steps + 1
+ * A violation step changes neither p, m nor v (Algorithm 1: theta_t = theta_{t-1})
+ * and does not advance t; a non-finite step changes nothing at all.
+ *
+ * gac_attach_adamw   binds the optimizer state of every tensor of the context's
+ *                    list (same order, same numel; float32 device buffers, CALLER-
+ *                    owned) and sets the number of updates applied so far
+ *                    (0 for a fresh optimizer).  Allocates a second table.
+ * gac_project_adamw  replaces gac_project for this step (same call order rules).
+ *                    Needs state_mode RAW.  opt is a host pointer, copied.
+ * Errors: INVALID_ARG, STATE (not attached, no decision pending), CUDA.
+ */
+typedef struct {
+    void *p;   /* parameter            */
+    void *m;   /* first moment         */
+    void *v;   /* second moment        */
+} gac_opt_tensor;
+typedef struct {
+    double lr, beta1, beta2, eps, weight_decay;
+} gac_adamw;
+void gac_default_adamw(gac_adamw *opt);   /* Table 2 values */
+int gac_attach_adamw(gac_ctx *ctx, const gac_opt_tensor *list, uint32_t n, uint64_t applied_steps);
+int gac_project_adamw(gac_ctx *ctx, void *cuda_stream, const gac_adamw *opt,
+                      const float *coef_override, gac_result *host_out);
 
 /* Releases what the context owns (never g or d).  NULL is accepted. */
 int gac_free(gac_ctx *ctx);

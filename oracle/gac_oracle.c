@@ -329,3 +329,55 @@ void orc_project(void *g, int g_dt, float *d, uint64_t n, const orc_hparams *hp,
         }                              /* ORC_STATE_HOLD: d unchanged */
     }
 }
+
+/* ---- the step after the path: GAC output consumed by AdamW --------------- */
+
+/* Algorithm 1 hands the (safe or projected) gradient to the optimizer; the
+ * paper trains with AdamW (Table 2: lr 1e-6, betas (0.9, 0.999), eps 1e-8,
+ * weight decay 1e-2).  This is the decoupled-weight-decay Adam of Loshchilov
+ * and Hutter as commonly implemented:
+ *     p <- p (1 - lr wd)
+ *     m <- b1 m + (1 - b1) g'          v <- b2 v + (1 - b2) g'^2
+ *     p <- p - (lr / (1 - b1^t)) m / (sqrt(v) / sqrt(1 - b2^t) + eps)
+ * with t the number of updates applied so far including this one, fed with the
+ * UNROUNDED g' = clip_scale (beta g + coef d) (projection) or clip_scale g
+ * (safe).  A skipped step (violation) leaves p, m, v alone: theta_t = theta_{t-1}.
+ * g itself is not written.  d is refreshed as in orc_project.  p, m, v are binary32. */
+typedef struct {
+    double lr, beta1, beta2, eps, weight_decay;
+} orc_adamw;
+
+void orc_project_adamw(const void *g, int g_dt, float *d, float *p, float *m, float *v, uint64_t n,
+                       const orc_hparams *hp, int regime, int nonfinite, float coef, int d_is_zero,
+                       double clip_scale, const orc_adamw *o, uint64_t t)
+{
+    if (nonfinite)
+        return;
+    double bc1 = 1.0 - pow(o->beta1, (double)t);
+    double bc2 = 1.0 - pow(o->beta2, (double)t);
+    double step_size = o->lr / bc1;
+    double sqrt_bc2 = sqrt(bc2);
+    for (uint64_t i = 0; i < n; ++i) {
+        double gi = elem_as_double(g, g_dt, i);
+        if (regime != ORC_VIOLATION) {
+            double gout = gi;
+            if (regime == ORC_PROJECT) {
+                double di = d_is_zero ? 0.0 : (double)d[i];
+                gout = hp->beta * gi + (double)coef * di;
+            }
+            if (clip_scale != 1.0)
+                gout = clip_scale * gout;
+            double pi = (double)p[i] * (1.0 - o->lr * o->weight_decay);
+            double mi = o->beta1 * (double)m[i] + (1.0 - o->beta1) * gout;
+            double vi = o->beta2 * (double)v[i] + (1.0 - o->beta2) * gout * gout;
+            double denom = sqrt(vi) / sqrt_bc2 + o->eps;
+            pi = pi - step_size * (mi / denom);
+            p[i] = (float)pi;
+            m[i] = (float)mi;
+            v[i] = (float)vi;
+        }
+        if (hp->state_mode == ORC_STATE_RAW)
+            d[i] = (float)gi;
+        /* other state modes are not offered by the fused form */
+    }
+}

@@ -56,6 +56,11 @@ class _HParams(ctypes.Structure):
                 ("clip_max_norm", ctypes.c_double), ("clip_eps", ctypes.c_double)]
 
 
+class _AdamW(ctypes.Structure):
+    _fields_ = [("lr", ctypes.c_double), ("beta1", ctypes.c_double), ("beta2", ctypes.c_double),
+                ("eps", ctypes.c_double), ("weight_decay", ctypes.c_double)]
+
+
 class _Decision(ctypes.Structure):
     _fields_ = [("dot", ctypes.c_double), ("gg", ctypes.c_double), ("dd", ctypes.c_double),
                 ("cosine", ctypes.c_double), ("alpha", ctypes.c_double),
@@ -86,6 +91,10 @@ def lib():
         L.orc_outgoing_sqnorm.restype = None
         L.orc_clip_scale.argtypes = [ctypes.c_double, ctypes.POINTER(_HParams)]
         L.orc_clip_scale.restype = ctypes.c_double
+        L.orc_project_adamw.argtypes = [vp, i32, vp, vp, vp, vp, u64, ctypes.POINTER(_HParams), i32,
+                                        i32, ctypes.c_float, i32, ctypes.c_double,
+                                        ctypes.POINTER(_AdamW), u64]
+        L.orc_project_adamw.restype = None
         L.orc_round_to_bf16.argtypes = [vp, vp, u64]
         for f in (L.orc_acc_init, L.orc_stats_accumulate, L.orc_acc_value, L.orc_acc_merge,
                   L.orc_stats_pairwise, L.orc_decide, L.orc_project, L.orc_round_to_bf16):
@@ -330,3 +339,44 @@ class RunningStats:
         out = (ctypes.c_double * 3)()
         lib().orc_acc_value(ctypes.byref(self._tot), out)
         return float(out[0]), float(out[1]), float(out[2])
+
+
+@dataclass
+class AdamW:
+    """AdamW hyper-parameters; defaults are the paper's (Table 2)."""
+    lr: float = 1e-6
+    beta1: float = 0.9
+    beta2: float = 0.999
+    eps: float = 1e-8
+    weight_decay: float = 1e-2
+
+    def c(self) -> _AdamW:
+        return _AdamW(self.lr, self.beta1, self.beta2, self.eps, self.weight_decay)
+
+
+def project_adamw(g_list, d_list, p_list, m_list, v_list, hp: HParams, dec: Decision, opt: AdamW,
+                  t: int, first_step: bool = False, coef: Optional[float] = None) -> bool:
+    """The GAC update consumed directly by AdamW (Algorithm 1's parameter update with
+    the optimizer of Table 2): p, m, v and the stored direction d change in place, g is
+    only read.  `t` is the number of updates applied so far including this one.
+    Returns True when the update was applied (False on a skipped step)."""
+    L = lib()
+    chp, copt = hp.c(), opt.c()
+    k = dec.coef if coef is None else float(np.float32(coef))
+    scale = 1.0
+    if hp.clip_max_norm > 0 and not dec.nonfinite and dec.regime != VIOLATION:
+        dec.out_norm = outgoing_norm(g_list, d_list, hp, dec, first_step, coef)
+        scale = float(L.orc_clip_scale(dec.out_norm ** 2, ctypes.byref(chp)))
+    dec.clip_scale = scale
+    for g, d, p, m, v in zip(g_list, d_list, p_list, m_list, v_list):
+        gp, gdt, n = _ptr_dt_n(g)
+        ptrs = []
+        for x in (d, p, m, v):
+            xp, xdt, xn = _ptr_dt_n(x)
+            if xdt != F32 or xn != n:
+                raise TypeError("d, p, m, v must be float32 of the gradient's length")
+            ptrs.append(xp)
+        L.orc_project_adamw(gp, gdt, ptrs[0], ptrs[1], ptrs[2], ptrs[3], n, ctypes.byref(chp),
+                            dec.regime, dec.nonfinite, ctypes.c_float(k), 1 if first_step else 0,
+                            ctypes.c_double(scale), ctypes.byref(copt), t)
+    return (not dec.nonfinite) and dec.regime != VIOLATION

@@ -42,10 +42,20 @@ class gac_result(ctypes.Structure):
                 ("cos", ctypes.c_double), ("alpha", ctypes.c_double), ("coef64", ctypes.c_double),
                 ("coef", ctypes.c_float), ("regime", ctypes.c_int32), ("nonfinite", ctypes.c_int32),
                 ("staleness", ctypes.c_uint32), ("step", ctypes.c_uint64),
-                ("out_norm", ctypes.c_double), ("clip_scale", ctypes.c_double)]
+                ("out_norm", ctypes.c_double), ("clip_scale", ctypes.c_double),
+                ("applied_steps", ctypes.c_uint64)]
 
     def as_dict(self):
         return {k: getattr(self, k) for k, _ in self._fields_}
+
+
+class gac_opt_tensor(ctypes.Structure):
+    _fields_ = [("p", ctypes.c_void_p), ("m", ctypes.c_void_p), ("v", ctypes.c_void_p)]
+
+
+class gac_adamw(ctypes.Structure):
+    _fields_ = [("lr", ctypes.c_double), ("beta1", ctypes.c_double), ("beta2", ctypes.c_double),
+                ("eps", ctypes.c_double), ("weight_decay", ctypes.c_double)]
 
 
 class gac_info(ctypes.Structure):
@@ -58,7 +68,7 @@ class gac_info(ctypes.Structure):
 
 EXPORTS = ["gac_default_hparams", "gac_init", "gac_stats", "gac_stats_partial", "gac_decide",
            "gac_project", "gac_free", "gac_last_error", "gac_set_launch", "gac_get_info",
-           "gac_stats_static"]
+           "gac_stats_static", "gac_default_adamw", "gac_attach_adamw", "gac_project_adamw"]
 
 _lib = None
 
@@ -96,6 +106,13 @@ def load_library() -> ctypes.CDLL:
     L.gac_stats_static.argtypes = [ctypes.POINTER(gac_tensor), u32, i32, i32,
                                    ctypes.POINTER(gac_hparams), u64, u32, i32, vp, vp]
     L.gac_stats_static.restype = i32
+    L.gac_default_adamw.argtypes = [ctypes.POINTER(gac_adamw)]
+    L.gac_default_adamw.restype = None
+    L.gac_attach_adamw.argtypes = [vp, ctypes.POINTER(gac_opt_tensor), u32, u64]
+    L.gac_attach_adamw.restype = i32
+    L.gac_project_adamw.argtypes = [vp, vp, ctypes.POINTER(gac_adamw), ctypes.POINTER(ctypes.c_float),
+                                    ctypes.POINTER(gac_result)]
+    L.gac_project_adamw.restype = i32
     for name in ("gac_init", "gac_stats", "gac_stats_partial", "gac_decide", "gac_project",
                  "gac_free", "gac_set_launch", "gac_get_info"):
         getattr(L, name).restype = i32
@@ -272,3 +289,45 @@ def result_from_tensor(t: torch.Tensor) -> gac_result:
     """Decodes a gac_result held in a uint8 tensor (copied to the host here)."""
     raw = bytes(t.detach().cpu().numpy().tobytes()[: ctypes.sizeof(gac_result)])
     return gac_result.from_buffer_copy(raw)
+
+
+@dataclass
+class AdamW:
+    """AdamW hyper-parameters; defaults are the paper's (Table 2)."""
+    lr: float = 1e-6
+    beta1: float = 0.9
+    beta2: float = 0.999
+    eps: float = 1e-8
+    weight_decay: float = 1e-2
+
+    def c(self) -> gac_adamw:
+        return gac_adamw(self.lr, self.beta1, self.beta2, self.eps, self.weight_decay)
+
+
+def gac_attach_adamw(ctx: GacContext, p_list: Sequence[torch.Tensor], m_list: Sequence[torch.Tensor],
+                     v_list: Sequence[torch.Tensor], applied_steps: int = 0) -> None:
+    """Binds float32 parameters and AdamW moments (one per tensor of the context's list)."""
+    n = len(p_list)
+    arr = (gac_opt_tensor * max(n, 1))()
+    for i, (p, m, v) in enumerate(zip(p_list, m_list, v_list)):
+        for t in (p, m, v):
+            if not (t.is_cuda and t.is_contiguous() and t.dtype == torch.float32):
+                raise ValueError("p, m, v must be contiguous float32 CUDA tensors")
+            if t.numel() != ctx._keep[0][i].numel():
+                raise ValueError(f"tensor {i}: optimizer state differs in numel from the gradient")
+        arr[i] = gac_opt_tensor(p.data_ptr(), m.data_ptr(), v.data_ptr())
+    ctx._check(load_library().gac_attach_adamw(ctx.handle, arr, n, applied_steps))
+    ctx._keep_opt = (list(p_list), list(m_list), list(v_list))
+
+
+def gac_project_adamw(ctx: GacContext, opt: AdamW, stream=None, coef_override: Optional[float] = None,
+                      fetch: bool = False) -> Optional[gac_result]:
+    L = load_library()
+    res = gac_result() if fetch else None
+    k = ctypes.c_float(coef_override) if coef_override is not None else None
+    copt = opt.c()
+    rc = L.gac_project_adamw(ctx.handle, _stream_ptr(stream), ctypes.byref(copt),
+                             ctypes.byref(k) if k is not None else None,
+                             ctypes.byref(res) if fetch else None)
+    ctx._check(rc, allow_nonfinite=True)
+    return res

@@ -86,6 +86,24 @@ namespace {
 #ifndef GAC_PROJ_MINB_BF16
 #define GAC_PROJ_MINB_BF16 1
 #endif
+#ifndef GAC_ADAMW_T_F32
+#define GAC_ADAMW_T_F32 1024
+#endif
+#ifndef GAC_ADAMW_U_F32
+#define GAC_ADAMW_U_F32 1
+#endif
+#ifndef GAC_ADAMW_C_F32
+#define GAC_ADAMW_C_F32 1
+#endif
+#ifndef GAC_ADAMW_T_BF16
+#define GAC_ADAMW_T_BF16 1024
+#endif
+#ifndef GAC_ADAMW_U_BF16
+#define GAC_ADAMW_U_BF16 1
+#endif
+#ifndef GAC_ADAMW_C_BF16
+#define GAC_ADAMW_C_BF16 1
+#endif
 #ifndef GAC_CHUNK
 #define GAC_CHUNK 16384
 #endif
@@ -181,6 +199,16 @@ struct StatsGeom<float> {
 template <>
 struct StatsGeom<bf16_t> {
     static constexpr int T = GAC_STATS_T_BF16, U = GAC_STATS_U_BF16, C = GAC_STATS_C_BF16, MINB = GAC_STATS_MINB_BF16;
+};
+template <typename GT>
+struct AdamGeom;
+template <>
+struct AdamGeom<float> {
+    static constexpr int T = GAC_ADAMW_T_F32, U = GAC_ADAMW_U_F32, C = GAC_ADAMW_C_F32;
+};
+template <>
+struct AdamGeom<bf16_t> {
+    static constexpr int T = GAC_ADAMW_T_BF16, U = GAC_ADAMW_U_BF16, C = GAC_ADAMW_C_BF16;
 };
 template <typename GT>
 struct ProjGeom;
@@ -473,12 +501,11 @@ __device__ __forceinline__ float rank_one(float g, float d, float k, double beta
 }
 __device__ __forceinline__ float scaled(float g, double s) { return __double2float_rn(__dmul_rn(s, double(g))); }
 
-template <typename GT, int GOP, int DOP, bool BETA1>
+template <typename GT, int GOP, int DOP, bool BETA1, int T, int U>
 __device__ __forceinline__ void project_chunk(const Chunk &ch, float k, double beta, double s) {
     void *g = reinterpret_cast<void *>(ch.g);
     void *d = reinterpret_cast<void *>(ch.d);
     const uint32_t tid = threadIdx.x;
-    constexpr int T = ProjGeom<GT>::T, U = ProjGeom<GT>::U;
     constexpr bool kReadG = (GOP == G_FMA) || (GOP == G_SCALE) || (DOP == D_RAW);
     constexpr bool kReadD = (GOP == G_FMA);
     if (ch.flags & kChunkAligned) {
@@ -550,7 +577,7 @@ template <typename GT, int GOP, int DOP, bool BETA1>
 __device__ __forceinline__ void project_walk(const Chunk *chunks, uint32_t n_chunks, float k,
                                              double beta, double s) {
     for (uint32_t c = blockIdx.x; c < n_chunks; c += gridDim.x)
-        project_chunk<GT, GOP, DOP, BETA1>(load_chunk(chunks, c), k, beta, s);
+        project_chunk<GT, GOP, DOP, BETA1, ProjGeom<GT>::T, ProjGeom<GT>::U>(load_chunk(chunks, c), k, beta, s);
 }
 
 // The regime is read from the device-resident record, so no host round trip
@@ -584,6 +611,185 @@ gac_project_kernel(const Chunk *__restrict__ chunks, uint32_t n_chunks, gac_resu
         project_walk<GT, G_SCALE, dop, true>(chunks, n_chunks, k, 1.0, s);   // safe step, clipped: g'' = s g
     } else if (STATE != GAC_STATE_HOLD) {
         project_walk<GT, G_KEEP, D_RAW, true>(chunks, n_chunks, k, 1.0, 1.0);   // d' = g, g untouched
+    }
+}
+
+// ------------------------------------------------ projection fused with AdamW
+
+struct __align__(16) OptChunk {
+    uint64_t p, m, v, pad;   // device addresses of the chunk's first parameter / moment elements
+};
+static_assert(sizeof(OptChunk) == 32, "optimizer chunk descriptors are read as two 16-byte words");
+
+struct AdamDev {
+    double lr, beta1, beta2, eps, weight_decay;
+};
+
+struct AdamConst {
+    double b1, c1, b2, c2;                       // moment recurrences
+    double step_size, inv_sqrt_bc2, eps, lr_wd;  // lr/(1-b1^t), 1/sqrt(1-b2^t), eps, lr*wd
+};
+
+// The outgoing gradient in binary64, unrounded: the moments are differences of
+// nearly equal terms often enough that a binary32 g' would cost them digits.
+template <int GOP>
+__device__ __forceinline__ double outgoing64(float g, float d, float k, double beta, double s) {
+    if (GOP == G_FMA)
+        return __dmul_rn(s, __dadd_rn(__dmul_rn(beta, double(g)), __dmul_rn(double(k), double(d))));
+    if (GOP == G_SCALE) return __dmul_rn(s, double(g));
+    return double(g);
+}
+
+// One element of: g' -> AdamW, in binary64 so that p - delta stays accurate
+// even where it cancels (tiny parameters).  The square root and the reciprocal
+// start from binary32 hardware results and take one Newton step each in
+// binary64 (relative error ~1e-14), far cheaper than the binary64 library
+// routines.  m, v and p are each rounded once on the way out.
+__device__ __forceinline__ void adamw_elem(double g64, float &p, float &m, float &v, const AdamConst &a) {
+    const double m64 = __dadd_rn(__dmul_rn(a.b1, double(m)), __dmul_rn(a.c1, g64));
+    const double v64 = __dadd_rn(__dmul_rn(a.b2, double(v)), __dmul_rn(__dmul_rn(a.c2, g64), g64));
+    double root = 0.0;
+    const float r32 = __fsqrt_rn(__double2float_rn(v64));
+    if (r32 > 0.0f) {
+        const double r = double(r32);
+        root = fma(fma(-r, r, v64), double(__fdividef(0.5f, r32)), r);   // r + (v - r^2)/(2r)
+    }
+    const double denom = fma(root, a.inv_sqrt_bc2, a.eps);
+    const double q = double(__frcp_rn(__double2float_rn(denom)));
+    const double inv = q * fma(-denom, q, 2.0);                           // q (2 - denom q)
+    const double delta = fma(a.lr_wd, double(p), a.step_size * (m64 * inv));
+    p = __double2float_rn(double(p) - delta);
+    m = __double2float_rn(m64);
+    v = __double2float_rn(v64);
+}
+
+template <typename GT, int GOP>
+__device__ __forceinline__ void adamw_chunk(const Chunk &ch, const OptChunk &oc, float k, double beta,
+                                            double s, const AdamConst &a) {
+    const void *g = reinterpret_cast<const void *>(ch.g);
+    void *d = reinterpret_cast<void *>(ch.d);
+    void *pp = reinterpret_cast<void *>(oc.p);
+    void *pm = reinterpret_cast<void *>(oc.m);
+    void *pv = reinterpret_cast<void *>(oc.v);
+    const uint32_t tid = threadIdx.x;
+    constexpr int T = AdamGeom<GT>::T, U = AdamGeom<GT>::U;
+    const bool vec = (ch.flags & kChunkAligned) && ((oc.p | oc.m | oc.v) % 16 == 0);
+    if (vec) {
+        const uint32_t nvec = ch.n >> 2;
+        for (uint32_t base = 0; base < nvec; base += T * U) {
+            F4 gv[U], dv[U], p4[U], m4[U], v4[U];
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+                const uint32_t w = base + u * T + tid;
+                dv[u] = F4{0.f, 0.f, 0.f, 0.f};
+                if (w < nvec) {
+                    gv[u] = Elem<GT>::template load4<GAC_LD_PROJECT>(g, w);
+                    if (GOP == G_FMA) dv[u] = Elem<float>::load4<GAC_LD_PROJECT>(d, w);
+                    p4[u] = Elem<float>::load4<GAC_LD_PROJECT>(pp, w);
+                    m4[u] = Elem<float>::load4<GAC_LD_PROJECT>(pm, w);
+                    v4[u] = Elem<float>::load4<GAC_LD_PROJECT>(pv, w);
+                }
+            }
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+                const uint32_t w = base + u * T + tid;
+                if (w >= nvec) continue;
+                float ge[4] = {gv[u].x, gv[u].y, gv[u].z, gv[u].w};
+                float pe[4] = {p4[u].x, p4[u].y, p4[u].z, p4[u].w};
+                float me[4] = {m4[u].x, m4[u].y, m4[u].z, m4[u].w};
+                float ve[4] = {v4[u].x, v4[u].y, v4[u].z, v4[u].w};
+                const float de[4] = {dv[u].x, dv[u].y, dv[u].z, dv[u].w};
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    adamw_elem(outgoing64<GOP>(ge[e], de[e], k, beta, s), pe[e], me[e], ve[e], a);
+                }
+                Elem<float>::store4(d, w, gv[u]);                       // d' = g, the raw gradient
+                Elem<float>::store4(pp, w, F4{pe[0], pe[1], pe[2], pe[3]});
+                Elem<float>::store4(pm, w, F4{me[0], me[1], me[2], me[3]});
+                Elem<float>::store4(pv, w, F4{ve[0], ve[1], ve[2], ve[3]});
+            }
+        }
+    }
+    const uint32_t first = vec ? ((ch.n >> 2) << 2) : 0u;
+    for (uint32_t i = first + tid; i < ch.n; i += T) {
+        const float x = Elem<GT>::load1(g, i);
+        const float dx = (GOP == G_FMA) ? Elem<float>::load1(d, i) : 0.f;
+        float pe = Elem<float>::load1(pp, i), me = Elem<float>::load1(pm, i), ve = Elem<float>::load1(pv, i);
+        adamw_elem(outgoing64<GOP>(x, dx, k, beta, s), pe, me, ve, a);
+        Elem<float>::store1(d, i, x);
+        Elem<float>::store1(pp, i, pe);
+        Elem<float>::store1(pm, i, me);
+        Elem<float>::store1(pv, i, ve);
+    }
+}
+
+__device__ __forceinline__ OptChunk load_opt_chunk(const OptChunk *table, uint32_t c) {
+    const uint4 *q = reinterpret_cast<const uint4 *>(table + c);
+    uint4 a = __ldg(q), b = __ldg(q + 1);
+    OptChunk oc;
+    oc.p = (uint64_t(a.y) << 32) | a.x;
+    oc.m = (uint64_t(a.w) << 32) | a.z;
+    oc.v = (uint64_t(b.y) << 32) | b.x;
+    oc.pad = 0;
+    return oc;
+}
+
+// Same decision logic as gac_project_kernel; a safe or projection step feeds
+// AdamW, a violation step only refreshes the stored direction.  The count of
+// applied updates lives in the decision record: every CTA reads it on entry,
+// and the last CTA to FINISH (arrival ticket, nobody waits) writes it back
+// incremented, so no CTA can see the new value during this launch.
+template <typename GT>
+__global__ void __launch_bounds__(AdamGeom<GT>::T, AdamGeom<GT>::C)
+gac_adamw_kernel(const Chunk *__restrict__ chunks, const OptChunk *__restrict__ opt_chunks,
+                 uint32_t n_chunks, gac_result *rec, unsigned *ticket, float coef_override,
+                 int use_override, double beta, double clip_max, double clip_eps, AdamDev o) {
+    if (rec->nonfinite) return;
+    const int regime = rec->regime;
+    const float k = use_override ? coef_override : rec->coef;
+    const unsigned long long t_prev = rec->applied_steps;
+    double s = 1.0;
+    if (clip_max > 0.0) {
+        double norm;
+        s = clip_factor(regime, rec->dot, rec->gg, rec->dd, beta, double(k), clip_max, clip_eps, &norm);
+        if (use_override && blockIdx.x == 0 && threadIdx.x == 0) {
+            rec->out_norm = norm;
+            rec->clip_scale = s;
+        }
+    }
+    const bool applies = (regime != GAC_REGIME_VIOLATION);
+    if (applies) {
+        const double t = double(t_prev + 1ull);
+        const double bc1 = 1.0 - pow(o.beta1, t), bc2 = 1.0 - pow(o.beta2, t);
+        AdamConst a;
+        a.b1 = o.beta1;
+        a.c1 = 1.0 - o.beta1;
+        a.b2 = o.beta2;
+        a.c2 = 1.0 - o.beta2;
+        a.step_size = o.lr / bc1;
+        a.inv_sqrt_bc2 = 1.0 / sqrt(bc2);
+        a.eps = o.eps;
+        a.lr_wd = o.lr * o.weight_decay;
+        for (uint32_t c = blockIdx.x; c < n_chunks; c += gridDim.x) {
+            const Chunk ch = load_chunk(chunks, c);
+            const OptChunk oc = load_opt_chunk(opt_chunks, c);
+            if (regime == GAC_REGIME_PROJECT) adamw_chunk<GT, G_FMA>(ch, oc, k, beta, s, a);
+            else if (s != 1.0) adamw_chunk<GT, G_SCALE>(ch, oc, k, 1.0, s, a);
+            else adamw_chunk<GT, G_KEEP>(ch, oc, k, 1.0, 1.0, a);
+        }
+    } else {
+        for (uint32_t c = blockIdx.x; c < n_chunks; c += gridDim.x)   // skipped step: d' = g only
+            project_chunk<GT, G_KEEP, D_RAW, true, AdamGeom<GT>::T, AdamGeom<GT>::U>(load_chunk(chunks, c), k, 1.0, 1.0);
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        __threadfence();
+        const unsigned done = atomicAdd(ticket, 1u);
+        if (done == gridDim.x - 1) {
+            rec->applied_steps = t_prev + (applies ? 1ull : 0ull);
+            __threadfence();
+            *ticket = 0u;
+        }
     }
 }
 
@@ -626,6 +832,9 @@ struct gac_ctx {
     int grid_stats = 0, grid_project = 0;
     int threads_stats = 0, threads_project = 0;
     const void *project_fn = nullptr;   // instantiation chosen from the hyper-parameters
+    OptChunk *d_opt_chunks = nullptr;   // optimizer state table of gac_attach_adamw
+    std::vector<gac_opt_tensor> opt_list;
+    int grid_adamw = 0, threads_adamw = 0;
 
     uint64_t last_projected_step = 0;
     uint64_t pending_step = 0;
@@ -671,6 +880,8 @@ size_t elem_size(int dt) { return dt == GAC_BF16 ? 2 : 4; }
 
 void release_device(gac_ctx *c) {
     if (c->d_chunks) cudaFree(c->d_chunks);
+    if (c->d_opt_chunks) cudaFree(c->d_opt_chunks);
+    c->d_opt_chunks = nullptr;
     if (c->d_partials) cudaFree(c->d_partials);
     if (c->d_ticket) cudaFree(c->d_ticket);
     if (c->d_rec) cudaFree(c->d_rec);
@@ -688,6 +899,37 @@ int resident_ctas(K kernel, int threads) {
     if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, kernel, threads, 0) != cudaSuccess || n < 1)
         n = 1;
     return std::min(n, kMaxCtasPerSm);
+}
+
+// Optimizer-state table parallel to the chunk table (same cuts), if state is attached.
+int build_opt_table(gac_ctx *c) {
+    if (c->d_opt_chunks) {
+        cudaFree(c->d_opt_chunks);
+        c->d_opt_chunks = nullptr;
+    }
+    if (c->opt_list.empty()) return GAC_OK;
+    const uint64_t ce = uint64_t(c->chunk_elems);
+    std::vector<OptChunk> table;
+    table.reserve(c->n_chunks);
+    for (size_t i = 0; i < c->list.size(); ++i) {
+        const gac_opt_tensor &o = c->opt_list[i];
+        for (uint64_t off = 0; off < c->list[i].numel; off += ce) {
+            OptChunk oc;
+            oc.p = reinterpret_cast<uint64_t>(o.p) + off * 4;
+            oc.m = reinterpret_cast<uint64_t>(o.m) + off * 4;
+            oc.v = reinterpret_cast<uint64_t>(o.v) + off * 4;
+            oc.pad = 0;
+            table.push_back(oc);
+        }
+    }
+    GAC_CUDA(c, cudaMalloc(&c->d_opt_chunks, table.size() * sizeof(OptChunk)));
+    GAC_CUDA(c, cudaMemcpy(c->d_opt_chunks, table.data(), table.size() * sizeof(OptChunk),
+                           cudaMemcpyHostToDevice));
+    const bool bf = (c->g_dt == GAC_BF16);
+    c->threads_adamw = bf ? AdamGeom<bf16_t>::T : AdamGeom<float>::T;
+    const int ctas = bf ? AdamGeom<bf16_t>::C : AdamGeom<float>::C;
+    c->grid_adamw = int(std::min<uint64_t>(uint64_t(c->sms) * ctas, c->n_chunks));
+    return GAC_OK;
 }
 
 // Cuts the list into chunks and uploads the table; sizes both grids.
@@ -745,7 +987,7 @@ int build_table(gac_ctx *c) {
     }
     c->grid_stats = int(std::min<uint64_t>(uint64_t(c->sms) * occ_s, c->n_chunks));
     c->grid_project = int(std::min<uint64_t>(uint64_t(c->sms) * occ_p, c->n_chunks));
-    return GAC_OK;
+    return build_opt_table(c);
 }
 
 int check_hparams(const gac_hparams *hp) {
@@ -963,6 +1205,69 @@ int gac_project(gac_ctx *ctx, void *cuda_stream, const float *coef_override, gac
     const uint32_t nc = uint32_t(ctx->n_chunks);
     reinterpret_cast<ProjectKernel>(const_cast<void *>(ctx->project_fn))<<<ctx->grid_project, ctx->threads_project, 0, s>>>(
         ctx->d_chunks, nc, ctx->d_rec, k, use, ctx->hp.beta, ctx->hp.clip_max_norm, ctx->hp.clip_eps);
+    GAC_CUDA(ctx, cudaGetLastError());
+    ++ctx->launches;
+    ctx->decision_ready = false;
+    ctx->last_projected_step = ctx->pending_step;
+    return host_out ? read_back(ctx, s, host_out) : GAC_OK;
+}
+
+void gac_default_adamw(gac_adamw *opt) {
+    if (!opt) return;
+    opt->lr = 1e-6;
+    opt->beta1 = 0.9;
+    opt->beta2 = 0.999;
+    opt->eps = 1e-8;
+    opt->weight_decay = 1e-2;
+}
+
+int gac_attach_adamw(gac_ctx *ctx, const gac_opt_tensor *list, uint32_t n, uint64_t applied_steps) {
+    if (!ctx) return fail(nullptr, GAC_ERR_INVALID_ARG, "ctx is NULL%s");
+    if (!list || n != ctx->list.size())
+        return fail(ctx, GAC_ERR_INVALID_ARG, "optimizer state list must have one entry per tensor of the context%s");
+    if (ctx->hp.state_mode != GAC_STATE_RAW)
+        return fail(ctx, GAC_ERR_INVALID_ARG, "the fused optimizer step needs state_mode RAW%s");
+    for (uint32_t i = 0; i < n; ++i) {
+        const void *ptrs[3] = {list[i].p, list[i].m, list[i].v};
+        for (const void *q : ptrs) {
+            if (!q) return fail(ctx, GAC_ERR_INVALID_ARG, "optimizer tensor %s%lld has a NULL pointer", "", i);
+            if (reinterpret_cast<uint64_t>(q) % 4)
+                return fail(ctx, GAC_ERR_INVALID_ARG, "optimizer tensor %s%lld is not element-aligned", "", i);
+        }
+    }
+    DeviceGuard guard(ctx->device);
+    ctx->opt_list.assign(list, list + n);
+    if (int rc = build_opt_table(ctx)) return rc;
+    const unsigned long long t0 = applied_steps;
+    GAC_CUDA(ctx, cudaMemcpy(&ctx->d_rec->applied_steps, &t0, sizeof(t0), cudaMemcpyHostToDevice));
+    return GAC_OK;
+}
+
+int gac_project_adamw(gac_ctx *ctx, void *cuda_stream, const gac_adamw *opt, const float *coef_override,
+                      gac_result *host_out) {
+    if (!ctx) return fail(nullptr, GAC_ERR_INVALID_ARG, "ctx is NULL%s");
+    if (!opt) return fail(ctx, GAC_ERR_INVALID_ARG, "opt is NULL%s");
+    if (!ctx->d_opt_chunks) return fail(ctx, GAC_ERR_STATE, "gac_project_adamw needs gac_attach_adamw first%s");
+    if (!ctx->decision_ready)
+        return fail(ctx, GAC_ERR_STATE, "gac_project_adamw needs the decision of gac_stats / gac_decide for this step%s");
+    if (!(opt->lr >= 0.0) || !(opt->beta1 >= 0.0 && opt->beta1 < 1.0) || !(opt->beta2 >= 0.0 && opt->beta2 < 1.0) ||
+        !(opt->eps >= 0.0) || !(opt->weight_decay >= 0.0) || !isfinite(opt->lr) || !isfinite(opt->eps) ||
+        !isfinite(opt->weight_decay))
+        return fail(ctx, GAC_ERR_INVALID_ARG, "AdamW needs lr, eps, weight_decay >= 0 and betas in [0,1)%s");
+    DeviceGuard guard(ctx->device);
+    cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+    const float k = coef_override ? *coef_override : 0.0f;
+    const int use = coef_override ? 1 : 0;
+    const uint32_t nc = uint32_t(ctx->n_chunks);
+    const AdamDev o{opt->lr, opt->beta1, opt->beta2, opt->eps, opt->weight_decay};
+    if (ctx->g_dt == GAC_BF16)
+        gac_adamw_kernel<bf16_t><<<ctx->grid_adamw, ctx->threads_adamw, 0, s>>>(
+            ctx->d_chunks, ctx->d_opt_chunks, nc, ctx->d_rec, ctx->d_ticket, k, use, ctx->hp.beta,
+            ctx->hp.clip_max_norm, ctx->hp.clip_eps, o);
+    else
+        gac_adamw_kernel<float><<<ctx->grid_adamw, ctx->threads_adamw, 0, s>>>(
+            ctx->d_chunks, ctx->d_opt_chunks, nc, ctx->d_rec, ctx->d_ticket, k, use, ctx->hp.beta,
+            ctx->hp.clip_max_norm, ctx->hp.clip_eps, o);
     GAC_CUDA(ctx, cudaGetLastError());
     ++ctx->launches;
     ctx->decision_ready = false;

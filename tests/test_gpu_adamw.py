@@ -1,0 +1,100 @@
+"""GPU parity of the fused GAC -> AdamW pass (Algorithm 1's parameter update with
+the optimizer of Table 2) against the CPU oracle, over consecutive steps that
+visit all three regimes."""
+import math
+
+import pytest
+import torch
+
+from oracle import gac_oracle as orc
+from paper_2603_01501_b200 import binding as gb
+from paper_2603_01501_b200 import synth
+
+from gpu_util import check_decision, check_sums, max_ulp, to_orc_hp
+
+pytestmark = pytest.mark.gpu
+
+
+def run_sequence(g_dtype, hp, opt_kw, shapes_name="mini", rhos=(None, 0.0, 0.3, 0.9, 0.2, 0.01, 0.5)):
+    shapes = synth.decoder_tensor_list(synth.DIMS[shapes_name])
+    sig = synth.per_tensor_scales(2, len(shapes))
+    gen = torch.Generator().manual_seed(7)
+    n_t = len(shapes)
+    p_cpu = [torch.randn(n, generator=gen) * 0.02 for _, n in shapes]
+    m_cpu = [torch.zeros(n) for _, n in shapes]
+    v_cpu = [torch.zeros(n) for _, n in shapes]
+    d_cpu = [torch.full((n,), float("nan")) for _, n in shapes]
+    g_gpu = [torch.empty(n, dtype=g_dtype, device="cuda") for _, n in shapes]
+    d_gpu = [t.cuda() for t in d_cpu]
+    p_gpu, m_gpu, v_gpu = ([t.cuda() for t in l] for l in (p_cpu, m_cpu, v_cpu))
+    ctx = gb.gac_init(g_gpu, d_gpu, hp)
+    gb.gac_attach_adamw(ctx, p_gpu, m_gpu, v_gpu, applied_steps=0)
+    gopt, oopt = gb.AdamW(**opt_kw), orc.AdamW(**opt_kw)
+    ohp = to_orc_hp(hp)
+    prev = [torch.randn(n, generator=gen) * s for (_, n), s in zip(shapes, sig)]
+    applied, regimes, worst = 0, [], 0
+    for t, rho in enumerate(rhos, start=1):
+        noise = [torch.randn(n, generator=gen) * s for (_, n), s in zip(shapes, sig)]
+        g = noise if rho is None else [rho * a + math.sqrt(1 - rho * rho) * b for a, b in zip(prev, noise)]
+        g = [x.to(g_dtype) for x in g]
+        prev = [x.float() for x in g]
+        for dst, src in zip(g_gpu, g):
+            dst.copy_(src)
+        first = t == 1
+        dec = orc.decide(orc.stats(g, d_cpu, first_step=first), ohp, first)
+        did = orc.project_adamw(g, d_cpu, p_cpu, m_cpu, v_cpu, ohp, dec, oopt, applied + 1, first)
+        applied += int(did)
+        res = gb.gac_stats(ctx, t)
+        after = gb.gac_project_adamw(ctx, gopt, coef_override=dec.coef if dec.regime == orc.PROJECT else None,
+                                     fetch=True)
+        check_sums(res, dec)
+        check_decision(res, dec)
+        assert after.applied_steps == applied
+        if hp.clip_max_norm > 0 and dec.regime != orc.VIOLATION:
+            assert abs(after.clip_scale - dec.clip_scale) <= 1e-9 * dec.clip_scale
+        for i in range(n_t):
+            assert torch.equal(g_gpu[i].cpu().view(torch.int16 if g_dtype == torch.bfloat16 else torch.int32),
+                               g[i].view(torch.int16 if g_dtype == torch.bfloat16 else torch.int32)), "g was written"
+            assert torch.equal(d_gpu[i].cpu(), d_cpu[i]), "stored direction is not the raw gradient"
+            for name, a, b in (("p", p_gpu[i], p_cpu[i]), ("m", m_gpu[i], m_cpu[i]), ("v", v_gpu[i], v_cpu[i])):
+                u = max_ulp(a.cpu(), b)
+                assert u <= 4, f"step {t} tensor {i} {name}: {u} ulp"
+                worst = max(worst, u)
+        regimes.append(dec.regime)
+    gb.gac_free(ctx)
+    return regimes, applied, worst
+
+
+@pytest.mark.parametrize("g_dtype", [torch.float32, torch.bfloat16], ids=["f32", "bf16"])
+def test_fused_adamw_paper_hyperparameters(g_dtype):
+    regimes, applied, _ = run_sequence(g_dtype, gb.HParams(), dict())        # Table 2 values
+    assert set(regimes) == {0, 1, 2}
+    assert applied == sum(r != gb.GAC_REGIME_VIOLATION for r in regimes)
+
+
+@pytest.mark.parametrize("hp,opt_kw", [
+    (gb.HParams(c_low=0.05, c_high=0.6, clip_max_norm=0.05), dict(lr=1e-3)),
+    (gb.HParams(c_low=0.05, c_high=0.6, clip_max_norm=1e6), dict(lr=1e-2, weight_decay=0.1)),
+    (gb.HParams(mode=gb.GAC_MODE_FIXED, alpha_fixed=0.25, beta=1.5), dict(lr=1e-3, beta1=0.8, beta2=0.95)),
+], ids=["clipped", "clip_inactive", "fixed_gains"])
+@pytest.mark.parametrize("g_dtype", [torch.float32, torch.bfloat16], ids=["f32", "bf16"])
+def test_fused_adamw_variants(hp, opt_kw, g_dtype):
+    run_sequence(g_dtype, hp, opt_kw)
+
+
+def test_fused_adamw_larger_list_and_call_rules():
+    run_sequence(torch.float32, gb.HParams(c_low=0.05, c_high=0.6), dict(lr=1e-4), shapes_name="small",
+                 rhos=(None, 0.3, 0.9))
+    g, d = [torch.ones(64, device="cuda")], [torch.ones(64, device="cuda") * 2]
+    ctx = gb.gac_init(g, d, gb.HParams())
+    gb.gac_stats(ctx, 2)
+    with pytest.raises(gb.GacError) as e:
+        gb.gac_project_adamw(ctx, gb.AdamW())
+    assert e.value.status == gb.GAC_ERR_STATE               # nothing attached
+    gb.gac_free(ctx)
+    ctx = gb.gac_init(g, d, gb.HParams(state_mode=gb.GAC_STATE_HOLD))
+    z = [torch.zeros(64, device="cuda")]
+    with pytest.raises(gb.GacError) as e:
+        gb.gac_attach_adamw(ctx, z, z, z)
+    assert e.value.status == gb.GAC_ERR_INVALID_ARG
+    gb.gac_free(ctx)

@@ -432,3 +432,66 @@ def test_clipping_closed_forms_and_regimes():
     dec = orc.step([g3], [d3], orc.HParams(clip_max_norm=1e-3))
     assert dec.regime == orc.VIOLATION and dec.clip_scale == 1.0
     np.testing.assert_array_equal(g3, (d * 3).astype(np.float32))
+
+
+# ---------------------------------------- the update consumed by AdamW (Table 2)
+
+def test_fused_adamw_matches_library_optimizer():
+    """Several consecutive steps of the oracle's GAC->AdamW against the unfused
+    route: oracle projection (kept in float64 by using float32-exact inputs) followed
+    by torch.optim.AdamW in float64."""
+    rng = np.random.default_rng(4)
+    n = 2000
+    opt = orc.AdamW(lr=1e-3, beta1=0.9, beta2=0.999, eps=1e-8, weight_decay=1e-2)
+    hp = orc.HParams(c_low=0.05, c_high=0.6)
+    p = rng.standard_normal(n).astype(np.float32)
+    m = np.zeros(n, np.float32)
+    v = np.zeros(n, np.float32)
+    d = np.zeros(n, np.float32)
+    tp = torch.nn.Parameter(torch.from_numpy(p.astype(np.float64)))
+    topt = torch.optim.AdamW([tp], lr=opt.lr, betas=(opt.beta1, opt.beta2), eps=opt.eps,
+                             weight_decay=opt.weight_decay)
+    t_applied = 0
+    prev = rng.standard_normal(n).astype(np.float32)
+    regimes = []
+    for step, rho in enumerate([None, 0.0, 0.3, 0.9, 0.2, 0.01], start=1):
+        noise = rng.standard_normal(n).astype(np.float32)
+        g = noise if rho is None else (rho * prev + math.sqrt(1 - rho * rho) * noise).astype(np.float32)
+        prev = g.copy()
+        first = step == 1
+        dec = orc.decide(orc.stats([g], [d], first_step=first), hp, first)
+        # unfused reference: g' from the definition in float64 (not rounded), then the library optimizer
+        gp = g.astype(np.float64)
+        if dec.regime == orc.PROJECT:
+            gp = hp.beta * gp + dec.coef * d.astype(np.float64)
+        applied = orc.project_adamw([g], [d], [p], [m], [v], hp, dec, opt, t_applied + 1, first)
+        regimes.append(dec.regime)
+        if applied:
+            t_applied += 1
+            # the library keeps float64 state, the oracle rounds p, m, v to float32 each step:
+            # restart the library from the oracle's rounded state so that one step is compared
+            tp.grad = torch.from_numpy(gp)
+            topt.step()
+            st = topt.state[tp]
+            np.testing.assert_allclose(m, st["exp_avg"].numpy(), rtol=1e-6, atol=1e-12)
+            np.testing.assert_allclose(v, st["exp_avg_sq"].numpy(), rtol=1e-6, atol=1e-14)
+            np.testing.assert_allclose(p, tp.detach().numpy(), rtol=1e-6, atol=1e-9)
+            with torch.no_grad():
+                tp.copy_(torch.from_numpy(p.astype(np.float64)))
+                st["exp_avg"].copy_(torch.from_numpy(m.astype(np.float64)))
+                st["exp_avg_sq"].copy_(torch.from_numpy(v.astype(np.float64)))
+        np.testing.assert_array_equal(d, g)
+    assert set(regimes) == {orc.SAFE, orc.PROJECT, orc.VIOLATION}
+    assert t_applied == regimes.count(orc.SAFE) + regimes.count(orc.PROJECT)
+
+
+def test_fused_adamw_skips_the_update_on_violation():
+    g = f32(1, 2, 3, 4)
+    d = f32(1, 2, 3, 4)
+    p, m, v = f32(5, 6, 7, 8), f32(.1, .2, .3, .4), f32(1, 1, 1, 1)
+    dec = orc.decide(orc.stats([g], [d]), orc.HParams())
+    assert dec.regime == orc.VIOLATION
+    applied = orc.project_adamw([g], [d * 2], [p], [m], [v], orc.HParams(), dec, orc.AdamW(), 1)
+    assert not applied
+    assert p.tolist() == [5, 6, 7, 8] and v.tolist() == [1, 1, 1, 1]
+    np.testing.assert_array_equal(m, f32(.1, .2, .3, .4))
