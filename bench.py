@@ -52,9 +52,10 @@ def measured_hbm_peak():
         return 6650.0, "fallback"
 
 
-def bytes_per_param(g_dtype) -> int:
+def bytes_per_param(g_dtype, d_dtype=torch.float32) -> int:
     sg = 2 if g_dtype == torch.bfloat16 else 4
-    return sg + 4
+    sd = 2 if d_dtype == torch.bfloat16 else 4
+    return sg + sd
 
 
 class ClockSampler:
@@ -149,6 +150,9 @@ class Workload:
         self.params = synth.list_numel(self.shapes)
         self.sigma = synth.per_tensor_scales(self.config_id, len(self.shapes))
         self.g, self.d = synth.gradient_list(self.shapes, self.rho, self.config_id, self.g_dtype, device)
+        self.d_dtype = synth.WORKLOAD_D_DTYPE.get(name, torch.float32)
+        if self.d_dtype != torch.float32:
+            self.d = [t.to(self.d_dtype) for t in self.d]
         self.scratch = torch.empty(max(n for _, n in self.shapes), dtype=torch.float32, device=device)
         self.gen = torch.Generator(device=device)
         self.gen.manual_seed(12345 + self.config_id)
@@ -231,10 +235,10 @@ def time_unchanged_regime(wl: Workload, steps: int):
     torch.cuda.synchronize()
     gb.gac_free(ctx)
     ms = sum(a.elapsed_time(b) for a, b in evs) / len(evs)
-    sg = 2 if wl.g_dtype == torch.bfloat16 else 4
-    nbytes = wl.params * ((sg + 4) + sg + 4)
+    bpp = 2 * bytes_per_param(wl.g_dtype, wl.d_dtype)
+    nbytes = wl.params * bpp
     return {"regime": gb.REGIME_NAMES[res.regime], "ms_per_step": ms,
-            "value": wl.params / (ms * 1e-3), "unit": UNIT, "bytes_per_param": (sg + 4) + sg + 4,
+            "value": wl.params / (ms * 1e-3), "unit": UNIT, "bytes_per_param": bpp,
             "hbm_gbs": nbytes / (ms * 1e-3) / 1e9}
 
 
@@ -415,11 +419,13 @@ def run_reference(args):
 def workload_config(name: str, wl):
     dims_key, g_dtype, rho, config_id = synth.WORKLOADS[name]
     shapes = synth.decoder_tensor_list(synth.DIMS[dims_key])
+    d_dtype = synth.WORKLOAD_D_DTYPE.get(name, torch.float32)
     return {"workload": f"{name}: {dims_key} decoder-shaped gradient list, "
-                        f"{'bf16' if g_dtype == torch.bfloat16 else 'f32'} g / f32 d, target cosine {rho}, "
+                        f"{'bf16' if g_dtype == torch.bfloat16 else 'f32'} g / "
+                        f"{'bf16' if d_dtype == torch.bfloat16 else 'f32'} d, target cosine {rho}, "
                         f"projection regime forced with c_low=0.05 c_high=2.0",
             "params_per_gpu": synth.list_numel(shapes), "tensors": len(shapes),
-            "bytes_per_param": 3 * bytes_per_param(g_dtype),
+            "bytes_per_param": 3 * bytes_per_param(g_dtype, d_dtype),
             "l2": "inputs larger than L2; a fresh gradient is written between timed steps",
             "timing": "per-step CUDA events around gac_stats+gac_project, summed over the timed steps"}
 
@@ -427,7 +433,7 @@ def workload_config(name: str, wl):
 # ------------------------------------------------------------------- driver
 
 def summarize(wl: Workload, s_ms, p_ms, peak, peak_kind):
-    bpp = bytes_per_param(wl.g_dtype)
+    bpp = bytes_per_param(wl.g_dtype, wl.d_dtype)
     s_avg, p_avg = sum(s_ms) / len(s_ms), sum(p_ms) / len(p_ms)
     step_ms = s_avg + p_avg
     proj_bytes = 2 * bpp * wl.params
@@ -436,6 +442,8 @@ def summarize(wl: Workload, s_ms, p_ms, peak, peak_kind):
     stats_gbs = stats_bytes / (s_avg * 1e-3) / 1e9
     tr_p, tr_s = recorded_traffic("gac_project_kernel"), recorded_traffic("gac_stats_kernel")
     key = "bf16" if wl.g_dtype == torch.bfloat16 else "f32"
+    if wl.d_dtype != torch.float32:
+        key += "_dbf16"
     return {
         "ms_per_step": step_ms, "stats_ms": s_avg, "project_ms": p_avg,
         "best_ms_per_step": min(a + b for a, b in zip(s_ms, p_ms)),

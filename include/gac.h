@@ -115,7 +115,9 @@ void gac_default_hparams(gac_hparams *hp);
  *   out          host pointer, receives the context
  *   list         host pointer to n entries (device pointers inside), copied
  *   n            number of tensors, >= 1; every numel >= 1
- *   g_dtype/d_dtype  supported pairs: (F32,F32), (BF16,F32)
+ *   g_dtype/d_dtype  supported pairs: (F32,F32), (BF16,F32), and (BF16,BF16) -- a
+ *                snapshot of half the size (App. A.2 "Memory footprint"), still an
+ *                exact copy of the bfloat16 gradient
  *   hp           host pointer; copied
  *   cuda_device  ordinal of the device that owns g and d
  * Allocates device and pinned memory (not capturable in a CUDA graph).

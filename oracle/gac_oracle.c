@@ -271,14 +271,14 @@ void orc_decide(const double sums[3], const orc_hparams *hp, int first_step, orc
  * clipping and before rounding: sum over i of (beta g_i + coef d_i)^2 in the
  * projection regime, of g_i^2 in the safe regime.  Accumulated into a->sum[0]
  * with Neumaier compensation so that a list can be fed tensor by tensor. */
-void orc_outgoing_sqnorm(orc_acc *a, const void *g, int g_dt, const float *d, uint64_t n,
+void orc_outgoing_sqnorm(orc_acc *a, const void *g, int g_dt, const void *d, int d_dt, uint64_t n,
                          const orc_hparams *hp, int regime, float coef, int d_is_zero)
 {
     for (uint64_t i = 0; i < n; ++i) {
         double gi = elem_as_double(g, g_dt, i);
         double out = gi;
         if (regime == ORC_PROJECT) {
-            double di = d_is_zero ? 0.0 : (double)d[i];
+            double di = d_is_zero ? 0.0 : elem_as_double(d, d_dt, i);
             out = hp->beta * gi + (double)coef * di;
         }
         neumaier_add(&a->sum[0], &a->comp[0], out * out);
@@ -295,11 +295,12 @@ double orc_clip_scale(double sqnorm, const orc_hparams *hp)
 }
 
 /* g (type g_dt) and d (binary32) are updated in place over n elements, given
- * the decision.  coef is the shared binary32 coefficient.  d_is_zero: d holds
+ * the decision.  d is binary32, or bfloat16 when g is bfloat16 (a snapshot of
+ * half the size).  coef is the shared binary32 coefficient.  d_is_zero: d holds
  * no valid data on the first step and is only written.  clip_scale (1 = none)
  * multiplies the outgoing gradient of a safe or projection step; a skipped
  * step sends nothing on, so it is not scaled. */
-void orc_project(void *g, int g_dt, float *d, uint64_t n, const orc_hparams *hp, int regime,
+void orc_project(void *g, int g_dt, void *d, int d_dt, uint64_t n, const orc_hparams *hp, int regime,
                  int nonfinite, float coef, int d_is_zero, double clip_scale)
 {
     if (nonfinite)
@@ -309,7 +310,7 @@ void orc_project(void *g, int g_dt, float *d, uint64_t n, const orc_hparams *hp,
         double gout = gi;
         int write_g = 0;
         if (regime == ORC_PROJECT) {
-            double di = d_is_zero ? 0.0 : (double)d[i];
+            double di = d_is_zero ? 0.0 : elem_as_double(d, d_dt, i);
             gout = hp->beta * gi + (double)coef * di;
             write_g = 1;
         } else if (regime == ORC_VIOLATION && hp->zero_on_violation) {
@@ -323,9 +324,9 @@ void orc_project(void *g, int g_dt, float *d, uint64_t n, const orc_hparams *hp,
         if (write_g)
             store_rounded(g, g_dt, i, gout);
         if (hp->state_mode == ORC_STATE_RAW) {
-            d[i] = (float)gi;          /* exact: gi came from <= 24 significant bits */
+            store_rounded(d, d_dt, i, gi);   /* exact whenever d is at least as wide as g */
         } else if (hp->state_mode == ORC_STATE_PROJECTED) {
-            d[i] = (float)elem_as_double(g, g_dt, i);
+            store_rounded(d, d_dt, i, elem_as_double(g, g_dt, i));
         }                              /* ORC_STATE_HOLD: d unchanged */
     }
 }
@@ -347,7 +348,7 @@ typedef struct {
     double lr, beta1, beta2, eps, weight_decay;
 } orc_adamw;
 
-void orc_project_adamw(const void *g, int g_dt, float *d, float *p, float *m, float *v, uint64_t n,
+void orc_project_adamw(const void *g, int g_dt, void *d, int d_dt, float *p, float *m, float *v, uint64_t n,
                        const orc_hparams *hp, int regime, int nonfinite, float coef, int d_is_zero,
                        double clip_scale, const orc_adamw *o, uint64_t t)
 {
@@ -362,7 +363,7 @@ void orc_project_adamw(const void *g, int g_dt, float *d, float *p, float *m, fl
         if (regime != ORC_VIOLATION) {
             double gout = gi;
             if (regime == ORC_PROJECT) {
-                double di = d_is_zero ? 0.0 : (double)d[i];
+                double di = d_is_zero ? 0.0 : elem_as_double(d, d_dt, i);
                 gout = hp->beta * gi + (double)coef * di;
             }
             if (clip_scale != 1.0)
@@ -377,7 +378,7 @@ void orc_project_adamw(const void *g, int g_dt, float *d, float *p, float *m, fl
             v[i] = (float)vi;
         }
         if (hp->state_mode == ORC_STATE_RAW)
-            d[i] = (float)gi;
+            store_rounded(d, d_dt, i, gi);
         /* other state modes are not offered by the fused form */
     }
 }

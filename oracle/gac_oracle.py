@@ -84,14 +84,14 @@ def lib():
         L.orc_stats_pairwise.argtypes = [vp, i32, vp, i32, u64, ctypes.c_double * 3]
         L.orc_decide.argtypes = [ctypes.c_double * 3, ctypes.POINTER(_HParams), i32,
                                  ctypes.POINTER(_Decision)]
-        L.orc_project.argtypes = [vp, i32, vp, u64, ctypes.POINTER(_HParams), i32, i32,
+        L.orc_project.argtypes = [vp, i32, vp, i32, u64, ctypes.POINTER(_HParams), i32, i32,
                                   ctypes.c_float, i32, ctypes.c_double]
-        L.orc_outgoing_sqnorm.argtypes = [ctypes.POINTER(_Acc), vp, i32, vp, u64,
+        L.orc_outgoing_sqnorm.argtypes = [ctypes.POINTER(_Acc), vp, i32, vp, i32, u64,
                                           ctypes.POINTER(_HParams), i32, ctypes.c_float, i32]
         L.orc_outgoing_sqnorm.restype = None
         L.orc_clip_scale.argtypes = [ctypes.c_double, ctypes.POINTER(_HParams)]
         L.orc_clip_scale.restype = ctypes.c_double
-        L.orc_project_adamw.argtypes = [vp, i32, vp, vp, vp, vp, u64, ctypes.POINTER(_HParams), i32,
+        L.orc_project_adamw.argtypes = [vp, i32, vp, i32, vp, vp, vp, u64, ctypes.POINTER(_HParams), i32,
                                         i32, ctypes.c_float, i32, ctypes.c_double,
                                         ctypes.POINTER(_AdamW), u64]
         L.orc_project_adamw.restype = None
@@ -243,8 +243,8 @@ def outgoing_norm(g_list: Sequence, d_list: Sequence, hp: HParams, dec: Decision
     L.orc_acc_init(ctypes.byref(acc))
     for g, d in zip(g_list, d_list):
         gp, gdt, n = _ptr_dt_n(g)
-        dp, _, _ = _ptr_dt_n(d)
-        L.orc_outgoing_sqnorm(ctypes.byref(acc), gp, gdt, dp, n, ctypes.byref(chp), dec.regime,
+        dp, ddt, _ = _ptr_dt_n(d)
+        L.orc_outgoing_sqnorm(ctypes.byref(acc), gp, gdt, dp, ddt, n, ctypes.byref(chp), dec.regime,
                               ctypes.c_float(k), 1 if first_step else 0)
     out = (ctypes.c_double * 3)()
     L.orc_acc_value(ctypes.byref(acc), out)
@@ -269,13 +269,14 @@ def project(g_list: Sequence, d_list: Sequence, hp: HParams, dec: Decision,
     for g, d in zip(g_list, d_list):
         gp, gdt, n = _ptr_dt_n(g)
         dp, ddt, nd = _ptr_dt_n(d)
-        if ddt != F32 or nd != n:
-            raise TypeError("stored direction must be float32 of the same length")
+        if nd != n or (ddt == BF16 and gdt != BF16):
+            raise TypeError("stored direction must be float32 (or bfloat16 with a bfloat16 gradient) "
+                            "of the gradient's length")
         for lo, hi in _ranges(n, threads):
-            jobs.append((gp + lo * _ELEM_BYTES[gdt], gdt, dp + lo * 4, hi - lo))
+            jobs.append((gp + lo * _ELEM_BYTES[gdt], gdt, dp + lo * _ELEM_BYTES[ddt], ddt, hi - lo))
 
     def run(job):
-        L.orc_project(job[0], job[1], job[2], job[3], ctypes.byref(chp), dec.regime,
+        L.orc_project(job[0], job[1], job[2], job[3], job[4], ctypes.byref(chp), dec.regime,
                       dec.nonfinite, ctypes.c_float(k), 1 if first_step else 0,
                       ctypes.c_double(scale))
 
@@ -370,13 +371,14 @@ def project_adamw(g_list, d_list, p_list, m_list, v_list, hp: HParams, dec: Deci
     dec.clip_scale = scale
     for g, d, p, m, v in zip(g_list, d_list, p_list, m_list, v_list):
         gp, gdt, n = _ptr_dt_n(g)
-        ptrs = []
-        for x in (d, p, m, v):
+        dp, ddt, dn = _ptr_dt_n(d)
+        ptrs = [dp]
+        for x in (p, m, v):
             xp, xdt, xn = _ptr_dt_n(x)
             if xdt != F32 or xn != n:
-                raise TypeError("d, p, m, v must be float32 of the gradient's length")
+                raise TypeError("p, m, v must be float32 of the gradient's length")
             ptrs.append(xp)
-        L.orc_project_adamw(gp, gdt, ptrs[0], ptrs[1], ptrs[2], ptrs[3], n, ctypes.byref(chp),
+        L.orc_project_adamw(gp, gdt, ptrs[0], ddt, ptrs[1], ptrs[2], ptrs[3], n, ctypes.byref(chp),
                             dec.regime, dec.nonfinite, ctypes.c_float(k), 1 if first_step else 0,
                             ctypes.c_double(scale), ctypes.byref(copt), t)
     return (not dec.nonfinite) and dec.regime != VIOLATION

@@ -190,6 +190,25 @@ struct bf16_t {
     uint16_t bits;
 };
 
+// Element-type pairs (gradient, stored direction).  A kernel's type parameter
+// is one of these tags: float = (binary32, binary32), bf16_t = (bfloat16,
+// binary32), bf16_pair_t = (bfloat16, bfloat16): a snapshot of half the size.
+struct bf16_pair_t {};
+template <typename P>
+struct PairOf {
+    using G = P;
+    using D = float;
+};
+template <>
+struct PairOf<bf16_pair_t> {
+    using G = bf16_t;
+    using D = bf16_t;
+};
+template <typename P>
+using GOf = typename PairOf<P>::G;
+template <typename P>
+using DOf = typename PairOf<P>::D;
+
 template <typename GT>
 struct StatsGeom;
 template <>
@@ -210,6 +229,10 @@ template <>
 struct AdamGeom<bf16_t> {
     static constexpr int T = GAC_ADAMW_T_BF16, U = GAC_ADAMW_U_BF16, C = GAC_ADAMW_C_BF16;
 };
+template <>
+struct StatsGeom<bf16_pair_t> : StatsGeom<bf16_t> {};
+template <>
+struct AdamGeom<bf16_pair_t> : AdamGeom<bf16_t> {};
 template <typename GT>
 struct ProjGeom;
 template <>
@@ -220,6 +243,8 @@ template <>
 struct ProjGeom<bf16_t> {
     static constexpr int T = GAC_PROJ_T_BF16, U = GAC_PROJ_U_BF16, C = GAC_PROJ_C_BF16, MINB = GAC_PROJ_MINB_BF16;
 };
+template <>
+struct ProjGeom<bf16_pair_t> : ProjGeom<bf16_t> {};
 
 __device__ __forceinline__ uint32_t pack_bf16x2_rn(float lo, float hi) {
     uint32_t r;
@@ -384,8 +409,8 @@ __device__ __forceinline__ void stats_chunk(const Chunk &ch, double &a_dot, doub
             for (int u = 0; u < U; ++u) {
                 const uint32_t v = base + u * T + tid;
                 if (v < nvec) {
-                    gv[u] = Elem<GT>::template load4<GAC_LD_STATS>(g, v);
-                    if (READ_D) dv[u] = Elem<float>::load4<GAC_LD_STATS>(d, v);
+                    gv[u] = Elem<GOf<GT>>::template load4<GAC_LD_STATS>(g, v);
+                    if (READ_D) dv[u] = Elem<DOf<GT>>::template load4<GAC_LD_STATS>(d, v);
                 } else {
                     gv[u] = F4{0.f, 0.f, 0.f, 0.f};
                     if (READ_D) dv[u] = F4{0.f, 0.f, 0.f, 0.f};
@@ -409,20 +434,20 @@ __device__ __forceinline__ void stats_chunk(const Chunk &ch, double &a_dot, doub
         }
         const uint32_t done = nvec << 2;
         if (tid < ch.n - done) {   // ragged tail of a tensor: < 4 elements
-            const double x = double(Elem<GT>::load1(g, done + tid));
+            const double x = double(Elem<GOf<GT>>::load1(g, done + tid));
             a_gg = fma(x, x, a_gg);
             if (READ_D) {
-                const double y = double(Elem<float>::load1(d, done + tid));
+                const double y = double(Elem<DOf<GT>>::load1(d, done + tid));
                 a_dot = fma(x, y, a_dot);
                 a_dd = fma(y, y, a_dd);
             }
         }
     } else {   // a base that is not 16-byte aligned: element-wise, still coalesced
         for (uint32_t i = tid; i < ch.n; i += T) {
-            const double x = double(Elem<GT>::load1(g, i));
+            const double x = double(Elem<GOf<GT>>::load1(g, i));
             a_gg = fma(x, x, a_gg);
             if (READ_D) {
-                const double y = double(Elem<float>::load1(d, i));
+                const double y = double(Elem<DOf<GT>>::load1(d, i));
                 a_dot = fma(x, y, a_dot);
                 a_dd = fma(y, y, a_dd);
             }
@@ -518,8 +543,8 @@ __device__ __forceinline__ void project_chunk(const Chunk &ch, float k, double b
                 gv[u] = F4{0.f, 0.f, 0.f, 0.f};
                 dv[u] = F4{0.f, 0.f, 0.f, 0.f};
                 if (v < nvec) {
-                    if (kReadG) gv[u] = Elem<GT>::template load4<GAC_LD_PROJECT>(g, v);
-                    if (kReadD) dv[u] = Elem<float>::load4<GAC_LD_PROJECT>(d, v);
+                    if (kReadG) gv[u] = Elem<GOf<GT>>::template load4<GAC_LD_PROJECT>(g, v);
+                    if (kReadD) dv[u] = Elem<DOf<GT>>::template load4<GAC_LD_PROJECT>(d, v);
                 }
             }
 #pragma unroll
@@ -535,39 +560,39 @@ __device__ __forceinline__ void project_chunk(const Chunk &ch, float k, double b
                     out.w = rank_one<BETA1>(gv[u].w, dv[u].w, k, beta, s);
                 }
                 if (GOP == G_SCALE) out = F4{scaled(gv[u].x, s), scaled(gv[u].y, s), scaled(gv[u].z, s), scaled(gv[u].w, s)};
-                if (GOP != G_KEEP) Elem<GT>::store4(g, v, out);
-                if (DOP == D_RAW) Elem<float>::store4(d, v, gv[u]);
+                if (GOP != G_KEEP) Elem<GOf<GT>>::store4(g, v, out);
+                if (DOP == D_RAW) Elem<DOf<GT>>::store4(d, v, gv[u]);
                 if (DOP == D_NEW) {
-                    if (GOP == G_FMA || GOP == G_SCALE) out = Elem<GT>::template load4<GAC_LD_PROJECT>(g, v);   // the value as stored (rounded)
-                    Elem<float>::store4(d, v, out);
+                    if (GOP == G_FMA || GOP == G_SCALE) out = Elem<GOf<GT>>::template load4<GAC_LD_PROJECT>(g, v);   // the value as stored (rounded)
+                    Elem<DOf<GT>>::store4(d, v, out);
                 }
             }
         }
         const uint32_t done = nvec << 2;
         if (tid < ch.n - done) {
             const uint32_t i = done + tid;
-            const float x = kReadG ? Elem<GT>::load1(g, i) : 0.f;
+            const float x = kReadG ? Elem<GOf<GT>>::load1(g, i) : 0.f;
             float out = (GOP == G_ZERO) ? 0.f : x;
-            if (GOP == G_FMA) out = rank_one<BETA1>(x, Elem<float>::load1(d, i), k, beta, s);
+            if (GOP == G_FMA) out = rank_one<BETA1>(x, Elem<DOf<GT>>::load1(d, i), k, beta, s);
             if (GOP == G_SCALE) out = scaled(x, s);
-            if (GOP != G_KEEP) Elem<GT>::store1(g, i, out);
-            if (DOP == D_RAW) Elem<float>::store1(d, i, x);
+            if (GOP != G_KEEP) Elem<GOf<GT>>::store1(g, i, out);
+            if (DOP == D_RAW) Elem<DOf<GT>>::store1(d, i, x);
             if (DOP == D_NEW) {
-                if (GOP == G_FMA || GOP == G_SCALE) out = Elem<GT>::load1(g, i);
-                Elem<float>::store1(d, i, out);
+                if (GOP == G_FMA || GOP == G_SCALE) out = Elem<GOf<GT>>::load1(g, i);
+                Elem<DOf<GT>>::store1(d, i, out);
             }
         }
     } else {
         for (uint32_t i = tid; i < ch.n; i += T) {
-            const float x = kReadG ? Elem<GT>::load1(g, i) : 0.f;
+            const float x = kReadG ? Elem<GOf<GT>>::load1(g, i) : 0.f;
             float out = (GOP == G_ZERO) ? 0.f : x;
-            if (GOP == G_FMA) out = rank_one<BETA1>(x, Elem<float>::load1(d, i), k, beta, s);
+            if (GOP == G_FMA) out = rank_one<BETA1>(x, Elem<DOf<GT>>::load1(d, i), k, beta, s);
             if (GOP == G_SCALE) out = scaled(x, s);
-            if (GOP != G_KEEP) Elem<GT>::store1(g, i, out);
-            if (DOP == D_RAW) Elem<float>::store1(d, i, x);
+            if (GOP != G_KEEP) Elem<GOf<GT>>::store1(g, i, out);
+            if (DOP == D_RAW) Elem<DOf<GT>>::store1(d, i, x);
             if (DOP == D_NEW) {
-                if (GOP == G_FMA || GOP == G_SCALE) out = Elem<GT>::load1(g, i);
-                Elem<float>::store1(d, i, out);
+                if (GOP == G_FMA || GOP == G_SCALE) out = Elem<GOf<GT>>::load1(g, i);
+                Elem<DOf<GT>>::store1(d, i, out);
             }
         }
     }
@@ -683,8 +708,8 @@ __device__ __forceinline__ void adamw_chunk(const Chunk &ch, const OptChunk &oc,
                 const uint32_t w = base + u * T + tid;
                 dv[u] = F4{0.f, 0.f, 0.f, 0.f};
                 if (w < nvec) {
-                    gv[u] = Elem<GT>::template load4<GAC_LD_PROJECT>(g, w);
-                    if (GOP == G_FMA) dv[u] = Elem<float>::load4<GAC_LD_PROJECT>(d, w);
+                    gv[u] = Elem<GOf<GT>>::template load4<GAC_LD_PROJECT>(g, w);
+                    if (GOP == G_FMA) dv[u] = Elem<DOf<GT>>::template load4<GAC_LD_PROJECT>(d, w);
                     p4[u] = Elem<float>::load4<GAC_LD_PROJECT>(pp, w);
                     m4[u] = Elem<float>::load4<GAC_LD_PROJECT>(pm, w);
                     v4[u] = Elem<float>::load4<GAC_LD_PROJECT>(pv, w);
@@ -703,7 +728,7 @@ __device__ __forceinline__ void adamw_chunk(const Chunk &ch, const OptChunk &oc,
                 for (int e = 0; e < 4; ++e) {
                     adamw_elem(outgoing64<GOP>(ge[e], de[e], k, beta, s), pe[e], me[e], ve[e], a);
                 }
-                Elem<float>::store4(d, w, gv[u]);                       // d' = g, the raw gradient
+                Elem<DOf<GT>>::store4(d, w, gv[u]);                       // d' = g, the raw gradient
                 Elem<float>::store4(pp, w, F4{pe[0], pe[1], pe[2], pe[3]});
                 Elem<float>::store4(pm, w, F4{me[0], me[1], me[2], me[3]});
                 Elem<float>::store4(pv, w, F4{ve[0], ve[1], ve[2], ve[3]});
@@ -712,11 +737,11 @@ __device__ __forceinline__ void adamw_chunk(const Chunk &ch, const OptChunk &oc,
     }
     const uint32_t first = vec ? ((ch.n >> 2) << 2) : 0u;
     for (uint32_t i = first + tid; i < ch.n; i += T) {
-        const float x = Elem<GT>::load1(g, i);
-        const float dx = (GOP == G_FMA) ? Elem<float>::load1(d, i) : 0.f;
+        const float x = Elem<GOf<GT>>::load1(g, i);
+        const float dx = (GOP == G_FMA) ? Elem<DOf<GT>>::load1(d, i) : 0.f;
         float pe = Elem<float>::load1(pp, i), me = Elem<float>::load1(pm, i), ve = Elem<float>::load1(pv, i);
         adamw_elem(outgoing64<GOP>(x, dx, k, beta, s), pe, me, ve, a);
-        Elem<float>::store1(d, i, x);
+        Elem<DOf<GT>>::store1(d, i, x);
         Elem<float>::store1(pp, i, pe);
         Elem<float>::store1(pm, i, me);
         Elem<float>::store1(pv, i, ve);
@@ -814,6 +839,7 @@ ProjectKernel pick_project(int state, bool beta1, bool zero) {
 struct gac_ctx {
     int device = 0;
     int g_dt = GAC_F32, d_dt = GAC_F32;
+    int pair = 0;   // PairId of (g_dt, d_dt)
     gac_hparams hp{};
     std::vector<gac_tensor> list;
     uint64_t total = 0;
@@ -901,6 +927,39 @@ int resident_ctas(K kernel, int threads) {
     return std::min(n, kMaxCtasPerSm);
 }
 
+// Supported element-type pairs and the kernels instantiated for them.
+enum PairId { kPairF32 = 0, kPairBf16F32 = 1, kPairBf16Bf16 = 2, kPairCount = 3 };
+
+int pair_id(int g_dt, int d_dt) {
+    if (g_dt == GAC_F32 && d_dt == GAC_F32) return kPairF32;
+    if (g_dt == GAC_BF16 && d_dt == GAC_F32) return kPairBf16F32;
+    if (g_dt == GAC_BF16 && d_dt == GAC_BF16) return kPairBf16Bf16;
+    return -1;
+}
+
+template <typename F>
+auto with_pair(int pair, F f) {
+    switch (pair) {
+        case kPairF32: return f(float{});
+        case kPairBf16F32: return f(bf16_t{});
+        default: return f(bf16_pair_t{});
+    }
+}
+
+using StatsKernel = void (*)(const Chunk *, uint32_t, double *, unsigned *, gac_result *, double *, DevHP);
+using AdamKernel = void (*)(const Chunk *, const OptChunk *, uint32_t, gac_result *, unsigned *, float, int,
+                            double, double, double, AdamDev);
+
+StatsKernel stats_kernel_of(int pair) {
+    return with_pair(pair, [](auto tag) -> StatsKernel { return gac_stats_kernel<decltype(tag)>; });
+}
+int stats_threads_of(int pair) {
+    return with_pair(pair, [](auto tag) { return StatsGeom<decltype(tag)>::T; });
+}
+int stats_cap_of(int pair) {
+    return with_pair(pair, [](auto tag) { return StatsGeom<decltype(tag)>::C; });
+}
+
 // Optimizer-state table parallel to the chunk table (same cuts), if state is attached.
 int build_opt_table(gac_ctx *c) {
     if (c->d_opt_chunks) {
@@ -925,9 +984,8 @@ int build_opt_table(gac_ctx *c) {
     GAC_CUDA(c, cudaMalloc(&c->d_opt_chunks, table.size() * sizeof(OptChunk)));
     GAC_CUDA(c, cudaMemcpy(c->d_opt_chunks, table.data(), table.size() * sizeof(OptChunk),
                            cudaMemcpyHostToDevice));
-    const bool bf = (c->g_dt == GAC_BF16);
-    c->threads_adamw = bf ? AdamGeom<bf16_t>::T : AdamGeom<float>::T;
-    const int ctas = bf ? AdamGeom<bf16_t>::C : AdamGeom<float>::C;
+    c->threads_adamw = with_pair(c->pair, [](auto tag) { return AdamGeom<decltype(tag)>::T; });
+    const int ctas = with_pair(c->pair, [](auto tag) { return AdamGeom<decltype(tag)>::C; });
     c->grid_adamw = int(std::min<uint64_t>(uint64_t(c->sms) * ctas, c->n_chunks));
     return GAC_OK;
 }
@@ -967,18 +1025,18 @@ int build_table(gac_ctx *c) {
                            cudaMemcpyHostToDevice));
     c->n_chunks = table.size();
 
-    const bool bf = (c->g_dt == GAC_BF16);
-    c->threads_stats = bf ? StatsGeom<bf16_t>::T : StatsGeom<float>::T;
-    c->threads_project = bf ? ProjGeom<bf16_t>::T : ProjGeom<float>::T;
-    int occ_s = bf ? resident_ctas(gac_stats_kernel<bf16_t>, c->threads_stats)
-                   : resident_ctas(gac_stats_kernel<float>, c->threads_stats);
+    c->threads_stats = stats_threads_of(c->pair);
+    c->threads_project = with_pair(c->pair, [](auto tag) { return ProjGeom<decltype(tag)>::T; });
+    int occ_s = resident_ctas(stats_kernel_of(c->pair), c->threads_stats);
     const bool beta1 = (c->hp.beta == 1.0), zero = (c->hp.zero_on_violation != 0);
-    ProjectKernel pk = c->g_dt == GAC_BF16 ? pick_project<bf16_t>(c->hp.state_mode, beta1, zero)
-                                           : pick_project<float>(c->hp.state_mode, beta1, zero);
+    const int state_mode = c->hp.state_mode;
+    ProjectKernel pk = with_pair(c->pair, [=](auto tag) -> ProjectKernel {
+        return pick_project<decltype(tag)>(state_mode, beta1, zero);
+    });
     c->project_fn = reinterpret_cast<const void *>(pk);
     int occ_p = resident_ctas(pk, c->threads_project);
-    const int cap_s = bf ? StatsGeom<bf16_t>::C : StatsGeom<float>::C;
-    const int cap_p = bf ? ProjGeom<bf16_t>::C : ProjGeom<float>::C;
+    const int cap_s = stats_cap_of(c->pair);
+    const int cap_p = with_pair(c->pair, [](auto tag) { return ProjGeom<decltype(tag)>::C; });
     if (cap_s > 0) occ_s = std::min(occ_s, cap_s);
     if (cap_p > 0) occ_p = std::min(occ_p, cap_p);
     if (c->ctas_per_sm > 0) {
@@ -1047,12 +1105,8 @@ int launch_stats(gac_ctx *c, uint64_t step, uint32_t staleness, cudaStream_t s, 
         return fail(c, GAC_ERR_STATE, "step %s%lld was already projected", "", (long long)step);
     const DevHP h = dev_hp(c, step, staleness, decide);
     const uint32_t nc = uint32_t(c->n_chunks);
-    if (c->g_dt == GAC_BF16)
-        gac_stats_kernel<bf16_t><<<c->grid_stats, c->threads_stats, 0, s>>>(c->d_chunks, nc, c->d_partials,
-                                                                    c->d_ticket, c->d_rec, sums_out, h);
-    else
-        gac_stats_kernel<float><<<c->grid_stats, c->threads_stats, 0, s>>>(c->d_chunks, nc, c->d_partials,
-                                                                   c->d_ticket, c->d_rec, sums_out, h);
+    stats_kernel_of(c->pair)<<<c->grid_stats, c->threads_stats, 0, s>>>(c->d_chunks, nc, c->d_partials, c->d_ticket,
+                                                                        c->d_rec, sums_out, h);
     GAC_CUDA(c, cudaGetLastError());
     ++c->launches;
     c->pending_step = step;
@@ -1082,8 +1136,8 @@ int gac_init(gac_ctx **out, const gac_tensor *list, uint32_t n, int g_dtype, int
     *out = nullptr;
     if (!list || n == 0) return fail(nullptr, GAC_ERR_INVALID_ARG, "empty tensor list%s");
     if (!hp) return fail(nullptr, GAC_ERR_INVALID_ARG, "hp is NULL%s");
-    if (!((g_dtype == GAC_F32 || g_dtype == GAC_BF16) && d_dtype == GAC_F32))
-        return fail(nullptr, GAC_ERR_DTYPE, "supported (g,d) element types: (f32,f32), (bf16,f32)%s");
+    if (pair_id(g_dtype, d_dtype) < 0)
+        return fail(nullptr, GAC_ERR_DTYPE, "supported (g,d) element types: (f32,f32), (bf16,f32), (bf16,bf16)%s");
     if (int rc = check_hparams(hp)) return rc;
     const size_t gs = elem_size(g_dtype), ds = elem_size(d_dtype);
     for (uint32_t i = 0; i < n; ++i) {
@@ -1111,6 +1165,7 @@ int gac_init(gac_ctx **out, const gac_tensor *list, uint32_t n, int g_dtype, int
     c->device = cuda_device;
     c->g_dt = g_dtype;
     c->d_dt = d_dtype;
+    c->pair = pair_id(g_dtype, d_dtype);
     c->hp = *hp;
     c->list.assign(list, list + n);
     for (uint32_t i = 0; i < n; ++i) c->total += list[i].numel;
@@ -1260,14 +1315,9 @@ int gac_project_adamw(gac_ctx *ctx, void *cuda_stream, const gac_adamw *opt, con
     const int use = coef_override ? 1 : 0;
     const uint32_t nc = uint32_t(ctx->n_chunks);
     const AdamDev o{opt->lr, opt->beta1, opt->beta2, opt->eps, opt->weight_decay};
-    if (ctx->g_dt == GAC_BF16)
-        gac_adamw_kernel<bf16_t><<<ctx->grid_adamw, ctx->threads_adamw, 0, s>>>(
-            ctx->d_chunks, ctx->d_opt_chunks, nc, ctx->d_rec, ctx->d_ticket, k, use, ctx->hp.beta,
-            ctx->hp.clip_max_norm, ctx->hp.clip_eps, o);
-    else
-        gac_adamw_kernel<float><<<ctx->grid_adamw, ctx->threads_adamw, 0, s>>>(
-            ctx->d_chunks, ctx->d_opt_chunks, nc, ctx->d_rec, ctx->d_ticket, k, use, ctx->hp.beta,
-            ctx->hp.clip_max_norm, ctx->hp.clip_eps, o);
+    const AdamKernel ak = with_pair(ctx->pair, [](auto tag) -> AdamKernel { return gac_adamw_kernel<decltype(tag)>; });
+    ak<<<ctx->grid_adamw, ctx->threads_adamw, 0, s>>>(ctx->d_chunks, ctx->d_opt_chunks, nc, ctx->d_rec, ctx->d_ticket,
+                                                      k, use, ctx->hp.beta, ctx->hp.clip_max_norm, ctx->hp.clip_eps, o);
     GAC_CUDA(ctx, cudaGetLastError());
     ++ctx->launches;
     ctx->decision_ready = false;
@@ -1327,7 +1377,7 @@ struct StaticSetup {
     bool ready = false;
     unsigned char *base = nullptr;   // DEVICE address of g_static_scratch on that device
     int sms = 0;
-    int occ_f32 = 0, occ_bf16 = 0;
+    int occ[kPairCount] = {0, 0, 0};
 };
 StaticSetup g_static_setup[kMaxDevices];
 std::mutex g_static_mutex;
@@ -1347,8 +1397,10 @@ int static_setup(int dev, StaticSetup **out) {
         if (e != cudaSuccess)
             return fail(nullptr, GAC_ERR_CUDA, "cudaDeviceGetAttribute failed: %s (CUDA error %lld)",
                         cudaGetErrorString(e), (long long)e);
-        st.occ_f32 = resident_ctas(gac_stats_kernel<float>, StatsGeom<float>::T);
-        st.occ_bf16 = resident_ctas(gac_stats_kernel<bf16_t>, StatsGeom<bf16_t>::T);
+        for (int pr = 0; pr < kPairCount; ++pr) {
+            st.occ[pr] = resident_ctas(stats_kernel_of(pr), stats_threads_of(pr));
+            if (stats_cap_of(pr) > 0) st.occ[pr] = std::min(st.occ[pr], stats_cap_of(pr));
+        }
         st.base = static_cast<unsigned char *>(ptr);
         st.ready = true;
     }
@@ -1365,8 +1417,8 @@ extern "C" int gac_stats_static(const gac_tensor *list, uint32_t n, int g_dtype,
     if (!hp) return fail(nullptr, GAC_ERR_INVALID_ARG, "hp is NULL%s");
     if (!result_dev) return fail(nullptr, GAC_ERR_INVALID_ARG, "result_dev is NULL%s");
     if (step == 0) return fail(nullptr, GAC_ERR_INVALID_ARG, "step counts from 1 (Algorithm 1)%s");
-    if (!((g_dtype == GAC_F32 || g_dtype == GAC_BF16) && d_dtype == GAC_F32))
-        return fail(nullptr, GAC_ERR_DTYPE, "supported (g,d) element types: (f32,f32), (bf16,f32)%s");
+    if (pair_id(g_dtype, d_dtype) < 0)
+        return fail(nullptr, GAC_ERR_DTYPE, "supported (g,d) element types: (f32,f32), (bf16,f32), (bf16,bf16)%s");
     if (int rc = check_hparams(hp)) return rc;
     if (cuda_device < 0 || cuda_device >= kMaxDevices)
         return fail(nullptr, GAC_ERR_INVALID_ARG, "cuda_device %s%lld out of range", "", cuda_device);
@@ -1421,14 +1473,11 @@ extern "C" int gac_stats_static(const gac_tensor *list, uint32_t n, int g_dtype,
     gac_ctx shell;            // only carries the hyper-parameters into dev_hp()
     shell.hp = *hp;
     const DevHP h = dev_hp(&shell, step, staleness, 1);
-    const int occ = g_dtype == GAC_BF16 ? st->occ_bf16 : st->occ_f32;
+    const int pair = pair_id(g_dtype, d_dtype);
+    const int occ = st->occ[pair];
     const uint32_t grid = uint32_t(std::min<uint64_t>(std::min<uint64_t>(uint64_t(st->sms) * occ, kStaticMaxCtas), n_chunks));
-    if (g_dtype == GAC_BF16)
-        gac_stats_kernel<bf16_t><<<grid, StatsGeom<bf16_t>::T, 0, s>>>(d_chunks, uint32_t(n_chunks), d_partials, d_ticket,
-                                                           result_dev, nullptr, h);
-    else
-        gac_stats_kernel<float><<<grid, StatsGeom<float>::T, 0, s>>>(d_chunks, uint32_t(n_chunks), d_partials, d_ticket,
-                                                          result_dev, nullptr, h);
+    stats_kernel_of(pair)<<<grid, stats_threads_of(pair), 0, s>>>(d_chunks, uint32_t(n_chunks), d_partials, d_ticket,
+                                                                  result_dev, nullptr, h);
     GAC_CUDA(nullptr, cudaGetLastError());
     return GAC_OK;
 }

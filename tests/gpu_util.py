@@ -77,10 +77,12 @@ def check_outputs(g_gpu, d_gpu, g_ref, d_ref, d_follows_g=False):
         assert u <= lim, f"tensor {i}: g' differs by {u} ulp (limit {lim})"
         worst = max(worst, u)
         if d_follows_g:
-            assert torch.equal(c, a.float()), f"tensor {i}: d' is not the stored g'"
+            assert torch.equal(c.float(), a.float()), f"tensor {i}: d' is not the stored g'"
             assert max_ulp(c.to(a.dtype), e.to(a.dtype)) <= lim
         else:
-            assert torch.equal(c.view(torch.int32), e.view(torch.int32)), f"tensor {i}: d' not bit-exact"
+            bits = torch.int32 if c.dtype == torch.float32 else torch.int16
+            assert c.dtype == e.dtype
+            assert torch.equal(c.view(bits), e.view(bits)), f"tensor {i}: d' not bit-exact"
     return worst
 
 

@@ -495,3 +495,25 @@ def test_fused_adamw_skips_the_update_on_violation():
     assert not applied
     assert p.tolist() == [5, 6, 7, 8] and v.tolist() == [1, 1, 1, 1]
     np.testing.assert_array_equal(m, f32(.1, .2, .3, .4))
+
+
+def test_bf16_snapshot_state():
+    """A bfloat16 stored direction next to a bfloat16 gradient: the refresh is an exact copy."""
+    torch.manual_seed(1)
+    d = (torch.randn(4000) * 0.01).to(torch.bfloat16)
+    g = (0.5 * d.float() + torch.randn(4000) * 0.01).to(torch.bfloat16)
+    g0, d0 = g.clone(), d.clone()
+    want = (dot64(g.float().numpy(), d.float().numpy()), dot64(g.float().numpy(), g.float().numpy()),
+            dot64(d.float().numpy(), d.float().numpy()))
+    got = orc.stats([g], [d])
+    for a, b in zip(got, want):
+        assert a == pytest.approx(b, rel=1e-15)
+    hp = orc.HParams(c_low=0.05, c_high=0.99, eps=0.0)
+    dec = orc.step([g], [d], hp)
+    assert dec.regime == orc.PROJECT and d.dtype == torch.bfloat16
+    assert torch.equal(d.view(torch.int16), g0.view(torch.int16))
+    x = g0.double().numpy() + dec.coef * d0.double().numpy()
+    ulp = 2.0 ** (np.floor(np.log2(np.abs(x))) - 7)
+    assert np.all(np.abs(g.double().numpy() - x) <= 0.5 * ulp * (1 + 1e-12))
+    with pytest.raises(TypeError):
+        orc.project([g0.float()], [d0], hp, dec)          # a float32 gradient needs a float32 snapshot
