@@ -86,6 +86,31 @@ namespace {
 #ifndef GAC_PROJ_MINB_BF16
 #define GAC_PROJ_MINB_BF16 1
 #endif
+// (bfloat16 g, bfloat16 d): half the bytes per vector of the mixed pair
+#ifndef GAC_STATS_T_BF16X
+#define GAC_STATS_T_BF16X GAC_STATS_T_BF16
+#endif
+#ifndef GAC_STATS_U_BF16X
+#define GAC_STATS_U_BF16X GAC_STATS_U_BF16
+#endif
+#ifndef GAC_STATS_C_BF16X
+#define GAC_STATS_C_BF16X GAC_STATS_C_BF16
+#endif
+#ifndef GAC_STATS_MINB_BF16X
+#define GAC_STATS_MINB_BF16X GAC_STATS_MINB_BF16
+#endif
+#ifndef GAC_PROJ_T_BF16X
+#define GAC_PROJ_T_BF16X GAC_PROJ_T_BF16
+#endif
+#ifndef GAC_PROJ_U_BF16X
+#define GAC_PROJ_U_BF16X 8
+#endif
+#ifndef GAC_PROJ_C_BF16X
+#define GAC_PROJ_C_BF16X GAC_PROJ_C_BF16
+#endif
+#ifndef GAC_PROJ_MINB_BF16X
+#define GAC_PROJ_MINB_BF16X GAC_PROJ_MINB_BF16
+#endif
 #ifndef GAC_ADAMW_T_F32
 #define GAC_ADAMW_T_F32 1024
 #endif
@@ -230,7 +255,9 @@ struct AdamGeom<bf16_t> {
     static constexpr int T = GAC_ADAMW_T_BF16, U = GAC_ADAMW_U_BF16, C = GAC_ADAMW_C_BF16;
 };
 template <>
-struct StatsGeom<bf16_pair_t> : StatsGeom<bf16_t> {};
+struct StatsGeom<bf16_pair_t> {
+    static constexpr int T = GAC_STATS_T_BF16X, U = GAC_STATS_U_BF16X, C = GAC_STATS_C_BF16X, MINB = GAC_STATS_MINB_BF16X;
+};
 template <>
 struct AdamGeom<bf16_pair_t> : AdamGeom<bf16_t> {};
 template <typename GT>
@@ -244,7 +271,9 @@ struct ProjGeom<bf16_t> {
     static constexpr int T = GAC_PROJ_T_BF16, U = GAC_PROJ_U_BF16, C = GAC_PROJ_C_BF16, MINB = GAC_PROJ_MINB_BF16;
 };
 template <>
-struct ProjGeom<bf16_pair_t> : ProjGeom<bf16_t> {};
+struct ProjGeom<bf16_pair_t> {
+    static constexpr int T = GAC_PROJ_T_BF16X, U = GAC_PROJ_U_BF16X, C = GAC_PROJ_C_BF16X, MINB = GAC_PROJ_MINB_BF16X;
+};
 
 __device__ __forceinline__ uint32_t pack_bf16x2_rn(float lo, float hi) {
     uint32_t r;
