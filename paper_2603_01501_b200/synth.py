@@ -43,6 +43,8 @@ DIMS: Dict[str, DecoderDims] = {
     # odd sizes on purpose so tensor tails are ragged
     # a 0.25 B list (1-2 GB per buffer): larger than L2, small enough for profiler captures
     "0.25b": DecoderDims(1024, 12, 8, 2, 128, 4096, 32000, False),
+    # one flat vector of 2^20 elements (a single "tensor"): the small, launch-bound case
+    "flat_1m": DecoderDims(0, 0, 0, 0, 0, 0, 0, True),
     "mini": DecoderDims(96, 3, 3, 1, 32, 250, 1021, True),
     "small": DecoderDims(384, 6, 6, 2, 64, 1030, 15013, False),
 }
@@ -51,6 +53,8 @@ DIMS: Dict[str, DecoderDims] = {
 def decoder_tensor_list(dims: DecoderDims) -> List[Tuple[str, int]]:
     """(name, numel) of every trainable tensor of a decoder-only transformer
     with grouped-query attention, SwiGLU MLP and RMSNorm, in module order."""
+    if dims.hidden == 0:
+        return [("flat", 1 << 20)]
     h, qd, kvd = dims.hidden, dims.q_heads * dims.head_dim, dims.kv_heads * dims.head_dim
     out: List[Tuple[str, int]] = [("embed", dims.vocab * h)]
     for l in range(dims.layers):
@@ -214,6 +218,7 @@ def refresh_gradient_list(g_list: Sequence[torch.Tensor], d_list: Sequence[torch
 
 WORKLOADS = {
     # name: (dims key, g dtype, rho, config id)  -- the decoder-shaped lists of the benchmark
+    "cfg1_flat_f32": ("flat_1m", torch.float32, 0.9, 1),
     "cfg2_1.5b_f32": ("1.5b", torch.float32, 0.8, 2),
     "cfg3_7b_bf16": ("7b", torch.bfloat16, 0.95, 3),
     "cfg5_14b_f32": ("14b", torch.float32, 0.9, 5),

@@ -342,3 +342,38 @@ def test_call_order_is_enforced():
     info = gb.gac_get_info(ctx)
     assert info.launches == 3 and info.total_elems == 100
     gb.gac_free(ctx)
+
+
+def test_step_can_be_captured_in_a_cuda_graph_and_replayed():
+    """With no host read-back both calls only enqueue kernels, so a step can be captured once and
+    replayed (the launch-bound case of small lists).  Replays must give what direct calls give."""
+    g_cpu, d_cpu = synth.flat_pair_with_cosine(1 << 20, 0.9, s=1.0, seed=0)
+    hp = gb.HParams(**FORCE)
+    g, d = [g_cpu.cuda()], [d_cpu.cuda()]
+    ctx = gb.gac_init(g, d, hp)
+    gb.gac_stats(ctx, 2, fetch=False)            # warm-up outside capture
+    gb.gac_project(ctx)
+    torch.cuda.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        graph.capture_begin()
+        gb.gac_stats(ctx, 3, fetch=False)
+        gb.gac_project(ctx)
+        graph.capture_end()
+    torch.cuda.current_stream().wait_stream(side)
+    for rho_seed in (1, 2):
+        g_new, d_new = synth.flat_pair_with_cosine(1 << 20, 0.5 + 0.2 * rho_seed, s=2.0, seed=rho_seed)
+        g[0].copy_(g_new)
+        d[0].copy_(d_new)
+        graph.replay()
+        torch.cuda.synchronize()
+        g_ref, d_ref = [g_new.clone()], [d_new.clone()]
+        dec = orc.step(g_ref, d_ref, to_orc_hp(hp))
+        # the coefficient is the library's own here (nothing can be overridden inside a replay)
+        assert dec.regime == orc.PROJECT
+        assert torch.equal(d[0].cpu(), d_ref[0])
+        assert max_ulp(g[0].cpu(), g_ref[0]) <= 64      # own coefficient: may differ in its last bit
+        assert float((g[0].cpu().double() - g_ref[0].double()).abs().max()) <= 2e-7 * float(g_new.abs().max())
+    gb.gac_free(ctx)
