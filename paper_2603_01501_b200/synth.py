@@ -224,10 +224,11 @@ WORKLOADS = {
     "cfg5_14b_f32": ("14b", torch.float32, 0.9, 5),
     "prof_0.25b_f32": ("0.25b", torch.float32, 0.9, 5),
     "prof_0.25b_bf16": ("0.25b", torch.bfloat16, 0.95, 3),
+    "prof_0.25b_bf16_dbf16": ("0.25b", torch.bfloat16, 0.95, 3),
     "cfg3_7b_bf16_dbf16": ("7b", torch.bfloat16, 0.95, 3),     # same list, bfloat16 snapshot
     "small_f32": ("small", torch.float32, 0.9, 2),
     "small_bf16": ("small", torch.bfloat16, 0.95, 3),
 }
 
 # element type of the stored direction where it is not float32
-WORKLOAD_D_DTYPE = {"cfg3_7b_bf16_dbf16": torch.bfloat16}
+WORKLOAD_D_DTYPE = {"cfg3_7b_bf16_dbf16": torch.bfloat16, "prof_0.25b_bf16_dbf16": torch.bfloat16}
