@@ -130,7 +130,7 @@ def recorded_traffic(kernel: str):
     try:
         with open(os.path.join(ROOT, "profiles", "traffic.json")) as fh:
             rec = json.load(fh)
-        src = os.path.join(ROOT, "paper_2603_01501_b200", "csrc", "gac.cu")
+        src = os.path.join(ROOT, "paper_2603_01501_b200", "csrc", "gac_kernels.cuh")
         if hashlib.sha256(open(src, "rb").read()).hexdigest() != rec["source_sha256"]:
             return None
         return rec["kernels"][kernel]
@@ -309,6 +309,17 @@ def check_regime(wl: Workload):
     gb.gac_project(wl.ctx)
     torch.cuda.synchronize()
     return res
+
+
+def e2e_fits_host(wl: Workload) -> bool:
+    """Every rank of the node pins its own host copy of the gradient list: do not
+    take more than half of the host's available memory."""
+    need = sum(t.numel() * t.element_size() for t in wl.g) * max(1, wl.world)
+    try:
+        import psutil
+        return need <= 0.5 * psutil.virtual_memory().available
+    except Exception:
+        return True
 
 
 def time_e2e(wl: Workload, steps: int, warmup: int):
@@ -535,15 +546,28 @@ def main():
     if world == 1 and args.adamw:
         line["fused_adamw"] = time_fused_adamw(wl, min(args.steps, 10))
     if not args.no_e2e:
-        try:
-            line["e2e"] = time_e2e(wl, min(args.steps, 5), 1)
+        # every rank takes the same branch: the decision to run is agreed on first, and the
+        # result is reduced by all ranks whether or not a rank failed
+        go = torch.tensor([1.0 if e2e_fits_host(wl) else 0.0], dtype=torch.float64, device=device)
+        if world > 1:
+            torch.distributed.all_reduce(go, op=torch.distributed.ReduceOp.MIN)
+        if float(go.item()) > 0:
+            try:
+                e2e = time_e2e(wl, min(args.steps, 5), 1)
+            except Exception as exc:
+                e2e = {"value": None, "unit": UNIT, "error": repr(exc)[:200], "ms_per_step": -1.0}
             if world > 1:
-                t = torch.tensor([line["e2e"]["ms_per_step"]], dtype=torch.float64, device=device)
+                t = torch.tensor([e2e["ms_per_step"], -e2e["ms_per_step"]], dtype=torch.float64, device=device)
                 torch.distributed.all_reduce(t, op=torch.distributed.ReduceOp.MAX)
-                line["e2e"]["ms_per_step"] = float(t.item())
-                line["e2e"]["value"] = wl.params * world / (float(t.item()) * 1e-3)
-        except Exception as exc:  # host memory too small for the pinned copy, ...
-            line["e2e"] = {"value": None, "unit": UNIT, "error": repr(exc)[:200]}
+                if -float(t[1].item()) < 0:       # some rank failed
+                    e2e = {"value": None, "unit": UNIT, "error": e2e.get("error", "a rank failed")}
+                else:
+                    e2e["ms_per_step"] = float(t[0].item())
+                    e2e["value"] = wl.params * world / (float(t[0].item()) * 1e-3)
+            line["e2e"] = e2e
+        else:
+            line["e2e"] = {"value": None, "unit": UNIT,
+                           "skipped": "the pinned host copies of all ranks would take more than half of the host's memory"}
     wl.close()
 
     if world == 1 and args.also != "none" and args.also != args.workload:

@@ -1,0 +1,847 @@
+// Device code of the GAC hot path for sm_100a: chunk descriptors, element
+// access for the supported element-type pairs, the fused triple reduction with
+// its fixed-order second stage and decision, the in-place projection with state
+// refresh, and the projection fused with AdamW.  Included by gac.cu only; the
+// host side of the C ABI lives there.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <math.h>
+#include <stdint.h>
+
+#include "gac.h"
+
+namespace {
+
+// Launch geometry.  Both kernels are bound by HBM, and on B200 their speed
+// depends on how many bytes each SM keeps in flight: too few starve the
+// memory system, too many make reads and write-backs of many chunks collide in
+// DRAM.  The macros exist so that variants can be built and timed side by side;
+// the defaults are the measured best per element type (T threads per CTA,
+// U four-element vectors in flight per thread and operand, C resident CTAs per
+// SM the grid is sized for with 0 = all that fit, MINB = occupancy asked of the
+// compiler with 0 = no request).
+#ifndef GAC_STATS_T_F32
+#define GAC_STATS_T_F32 256
+#endif
+#ifndef GAC_STATS_U_F32
+#define GAC_STATS_U_F32 8
+#endif
+#ifndef GAC_STATS_C_F32
+#define GAC_STATS_C_F32 0
+#endif
+#ifndef GAC_STATS_MINB_F32
+#define GAC_STATS_MINB_F32 4
+#endif
+#ifndef GAC_STATS_T_BF16
+#define GAC_STATS_T_BF16 256
+#endif
+#ifndef GAC_STATS_U_BF16
+#define GAC_STATS_U_BF16 8
+#endif
+#ifndef GAC_STATS_C_BF16
+#define GAC_STATS_C_BF16 0
+#endif
+#ifndef GAC_STATS_MINB_BF16
+#define GAC_STATS_MINB_BF16 4
+#endif
+#ifndef GAC_PROJ_T_F32
+#define GAC_PROJ_T_F32 256
+#endif
+#ifndef GAC_PROJ_U_F32
+#define GAC_PROJ_U_F32 8
+#endif
+#ifndef GAC_PROJ_C_F32
+#define GAC_PROJ_C_F32 1
+#endif
+#ifndef GAC_PROJ_MINB_F32
+#define GAC_PROJ_MINB_F32 1
+#endif
+#ifndef GAC_PROJ_T_BF16
+#define GAC_PROJ_T_BF16 512
+#endif
+#ifndef GAC_PROJ_U_BF16
+#define GAC_PROJ_U_BF16 4
+#endif
+#ifndef GAC_PROJ_C_BF16
+#define GAC_PROJ_C_BF16 1
+#endif
+#ifndef GAC_PROJ_MINB_BF16
+#define GAC_PROJ_MINB_BF16 1
+#endif
+// (bfloat16 g, bfloat16 d): half the bytes per vector of the mixed pair
+#ifndef GAC_STATS_T_BF16X
+#define GAC_STATS_T_BF16X GAC_STATS_T_BF16
+#endif
+#ifndef GAC_STATS_U_BF16X
+#define GAC_STATS_U_BF16X GAC_STATS_U_BF16
+#endif
+#ifndef GAC_STATS_C_BF16X
+#define GAC_STATS_C_BF16X GAC_STATS_C_BF16
+#endif
+#ifndef GAC_STATS_MINB_BF16X
+#define GAC_STATS_MINB_BF16X GAC_STATS_MINB_BF16
+#endif
+#ifndef GAC_PROJ_T_BF16X
+#define GAC_PROJ_T_BF16X GAC_PROJ_T_BF16
+#endif
+#ifndef GAC_PROJ_U_BF16X
+#define GAC_PROJ_U_BF16X 8
+#endif
+#ifndef GAC_PROJ_C_BF16X
+#define GAC_PROJ_C_BF16X GAC_PROJ_C_BF16
+#endif
+#ifndef GAC_PROJ_MINB_BF16X
+#define GAC_PROJ_MINB_BF16X GAC_PROJ_MINB_BF16
+#endif
+#ifndef GAC_ADAMW_T_F32
+#define GAC_ADAMW_T_F32 1024
+#endif
+#ifndef GAC_ADAMW_U_F32
+#define GAC_ADAMW_U_F32 1
+#endif
+#ifndef GAC_ADAMW_C_F32
+#define GAC_ADAMW_C_F32 1
+#endif
+#ifndef GAC_ADAMW_T_BF16
+#define GAC_ADAMW_T_BF16 1024
+#endif
+#ifndef GAC_ADAMW_U_BF16
+#define GAC_ADAMW_U_BF16 1
+#endif
+#ifndef GAC_ADAMW_C_BF16
+#define GAC_ADAMW_C_BF16 1
+#endif
+#ifndef GAC_CHUNK
+#define GAC_CHUNK 16384
+#endif
+// load flavour: 0 plain ld.global, 1 streaming (ld.global.cs), 2 read-only path (ld.global.nc)
+#ifndef GAC_LD_STATS
+#define GAC_LD_STATS 0
+#endif
+#ifndef GAC_LD_PROJECT
+#define GAC_LD_PROJECT 0
+#endif
+#ifndef GAC_ST      // 0 plain st.global, 1 streaming (st.global.cs), 2 write-through (st.global.wt)
+#define GAC_ST 1
+#endif
+constexpr int kDefaultChunk = GAC_CHUNK; // elements per chunk
+constexpr int kMaxCtasPerSm = 16;
+
+constexpr uint32_t kChunkAligned = 1u;  // both bases 16-byte aligned: vector path
+
+struct __align__(16) Chunk {
+    uint64_t g;      // device address of the chunk's first g element
+    uint64_t d;      // device address of the chunk's first d element
+    uint32_t n;      // elements in the chunk (<= chunk_elems)
+    uint32_t flags;
+    uint64_t pad;
+};
+static_assert(sizeof(Chunk) == 32, "chunk descriptors are read as two 16-byte words");
+
+// Hyper-parameters as the kernels see them.
+struct DevHP {
+    double c_low, c_high, eps, beta, alpha_fixed;
+    int mode, state_mode, zero_on_violation, first_step;
+    unsigned long long step;
+    unsigned staleness;
+    int decide;      // 0: only publish the three sums (sharded form)
+    double clip_max, clip_eps;
+};
+
+struct F4 {
+    float x, y, z, w;
+};
+
+// ---------------------------------------------------------------- element I/O
+
+template <int LD, typename V>
+__device__ __forceinline__ V ld_vec(const V *p) {
+    if (LD == 1) return __ldcs(p);
+    if (LD == 2) return __ldg(p);
+    return *p;
+}
+template <typename V>
+__device__ __forceinline__ void st_vec(V *p, V v) {
+#if GAC_ST == 1
+    __stcs(p, v);
+#elif GAC_ST == 2
+    __stwt(p, v);
+#else
+    *p = v;
+#endif
+}
+
+template <typename GT>
+struct Elem;
+
+template <>
+struct Elem<float> {
+    template <int LD>
+    static __device__ __forceinline__ F4 load4(const void *base, uint32_t v) {
+        float4 t = ld_vec<LD>(reinterpret_cast<const float4 *>(base) + v);
+        return F4{t.x, t.y, t.z, t.w};
+    }
+    static __device__ __forceinline__ void store4(void *base, uint32_t v, F4 a) {
+        st_vec(reinterpret_cast<float4 *>(base) + v, make_float4(a.x, a.y, a.z, a.w));
+    }
+    static __device__ __forceinline__ float load1(const void *base, uint32_t i) {
+        return reinterpret_cast<const float *>(base)[i];
+    }
+    static __device__ __forceinline__ void store1(void *base, uint32_t i, float a) {
+        reinterpret_cast<float *>(base)[i] = a;
+    }
+};
+
+// bfloat16 = the upper 16 bits of a binary32 pattern.
+struct bf16_t {
+    uint16_t bits;
+};
+
+// Element-type pairs (gradient, stored direction).  A kernel's type parameter
+// is one of these tags: float = (binary32, binary32), bf16_t = (bfloat16,
+// binary32), bf16_pair_t = (bfloat16, bfloat16): a snapshot of half the size.
+struct bf16_pair_t {};
+template <typename P>
+struct PairOf {
+    using G = P;
+    using D = float;
+};
+template <>
+struct PairOf<bf16_pair_t> {
+    using G = bf16_t;
+    using D = bf16_t;
+};
+template <typename P>
+using GOf = typename PairOf<P>::G;
+template <typename P>
+using DOf = typename PairOf<P>::D;
+
+template <typename GT>
+struct StatsGeom;
+template <>
+struct StatsGeom<float> {
+    static constexpr int T = GAC_STATS_T_F32, U = GAC_STATS_U_F32, C = GAC_STATS_C_F32, MINB = GAC_STATS_MINB_F32;
+};
+template <>
+struct StatsGeom<bf16_t> {
+    static constexpr int T = GAC_STATS_T_BF16, U = GAC_STATS_U_BF16, C = GAC_STATS_C_BF16, MINB = GAC_STATS_MINB_BF16;
+};
+template <typename GT>
+struct AdamGeom;
+template <>
+struct AdamGeom<float> {
+    static constexpr int T = GAC_ADAMW_T_F32, U = GAC_ADAMW_U_F32, C = GAC_ADAMW_C_F32;
+};
+template <>
+struct AdamGeom<bf16_t> {
+    static constexpr int T = GAC_ADAMW_T_BF16, U = GAC_ADAMW_U_BF16, C = GAC_ADAMW_C_BF16;
+};
+template <>
+struct StatsGeom<bf16_pair_t> {
+    static constexpr int T = GAC_STATS_T_BF16X, U = GAC_STATS_U_BF16X, C = GAC_STATS_C_BF16X, MINB = GAC_STATS_MINB_BF16X;
+};
+template <>
+struct AdamGeom<bf16_pair_t> : AdamGeom<bf16_t> {};
+template <typename GT>
+struct ProjGeom;
+template <>
+struct ProjGeom<float> {
+    static constexpr int T = GAC_PROJ_T_F32, U = GAC_PROJ_U_F32, C = GAC_PROJ_C_F32, MINB = GAC_PROJ_MINB_F32;
+};
+template <>
+struct ProjGeom<bf16_t> {
+    static constexpr int T = GAC_PROJ_T_BF16, U = GAC_PROJ_U_BF16, C = GAC_PROJ_C_BF16, MINB = GAC_PROJ_MINB_BF16;
+};
+template <>
+struct ProjGeom<bf16_pair_t> {
+    static constexpr int T = GAC_PROJ_T_BF16X, U = GAC_PROJ_U_BF16X, C = GAC_PROJ_C_BF16X, MINB = GAC_PROJ_MINB_BF16X;
+};
+
+__device__ __forceinline__ uint32_t pack_bf16x2_rn(float lo, float hi) {
+    uint32_t r;
+    asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
+    return r;
+}
+
+template <>
+struct Elem<bf16_t> {
+    template <int LD>
+    static __device__ __forceinline__ F4 load4(const void *base, uint32_t v) {
+        uint2 t = ld_vec<LD>(reinterpret_cast<const uint2 *>(base) + v);
+        return F4{__uint_as_float(t.x << 16), __uint_as_float(t.x & 0xFFFF0000u),
+                  __uint_as_float(t.y << 16), __uint_as_float(t.y & 0xFFFF0000u)};
+    }
+    static __device__ __forceinline__ void store4(void *base, uint32_t v, F4 a) {
+        st_vec(reinterpret_cast<uint2 *>(base) + v,
+               make_uint2(pack_bf16x2_rn(a.x, a.y), pack_bf16x2_rn(a.z, a.w)));
+    }
+    static __device__ __forceinline__ float load1(const void *base, uint32_t i) {
+        return __uint_as_float(uint32_t(reinterpret_cast<const uint16_t *>(base)[i]) << 16);
+    }
+    static __device__ __forceinline__ void store1(void *base, uint32_t i, float a) {
+        reinterpret_cast<uint16_t *>(base)[i] = uint16_t(pack_bf16x2_rn(a, 0.0f) & 0xFFFFu);
+    }
+};
+
+__device__ __forceinline__ Chunk load_chunk(const Chunk *table, uint32_t c) {
+    const uint4 *p = reinterpret_cast<const uint4 *>(table + c);
+    uint4 a = __ldg(p), b = __ldg(p + 1);
+    Chunk ch;
+    ch.g = (uint64_t(a.y) << 32) | a.x;
+    ch.d = (uint64_t(a.w) << 32) | a.z;
+    ch.n = b.x;
+    ch.flags = b.y;
+    ch.pad = 0;
+    return ch;
+}
+
+// ------------------------------------------------------- decision (O(1) work)
+
+// Global-norm clipping folded into the update (Table 2: "Gradient clipping
+// True").  The squared norm of what a step sends on follows from the three
+// sums alone: |beta g + k d|^2 = beta^2 <g,g> + 2 beta k <g,d> + k^2 <d,d> in the
+// projection regime (k = the binary32 coefficient actually applied), <g,g> in
+// the safe regime; a skipped step sends nothing on.  Factor as in the usual
+// global-norm clip: min(1, max_norm / (norm + clip_eps)).
+__device__ __forceinline__ double clip_factor(int regime, double dot, double gg, double dd, double beta,
+                                              double k, double clip_max, double clip_eps, double *norm_out) {
+    double n2 = gg;
+    if (regime == GAC_REGIME_PROJECT)
+        n2 = __dadd_rn(__dadd_rn(__dmul_rn(__dmul_rn(beta, beta), gg),
+                                 __dmul_rn(__dmul_rn(2.0 * beta, k), dot)),
+                       __dmul_rn(__dmul_rn(k, k), dd));
+    const double norm = __dsqrt_rn(fmax(n2, 0.0));
+    *norm_out = norm;
+    if (!(clip_max > 0.0) || regime == GAC_REGIME_VIOLATION) return 1.0;
+    const double f = __ddiv_rn(clip_max, __dadd_rn(norm, clip_eps));
+    return f < 1.0 ? f : 1.0;
+}
+
+// Cosine with eps outside the root (App. A.1), the inclusive branches of
+// Algorithm 1, alpha = c_low/|c| (Eq. 5) or the caller's gain (Eq. 3), and the
+// multiplier of d in the rank-one form of App. A.2.
+__device__ void take_decision(double dot, double gg, double dd, const DevHP &hp, gac_result *r) {
+    if (hp.first_step) {   // Algorithm 1: g_0 = 0
+        dot = 0.0;
+        dd = 0.0;
+    }
+    r->dot = dot;
+    r->gg = gg;
+    r->dd = dd;
+    r->alpha = 1.0;
+    r->coef64 = 0.0;
+    r->coef = 0.0f;
+    r->out_norm = 0.0;
+    r->clip_scale = 1.0;
+    r->staleness = hp.staleness;
+    r->step = hp.step;
+    r->nonfinite = !(isfinite(dot) && isfinite(gg) && isfinite(dd));
+    if (r->nonfinite) {
+        r->cos = __longlong_as_double(0x7FF8000000000000LL);
+        r->regime = GAC_REGIME_VIOLATION;
+        return;
+    }
+    if (gg == 0.0 || dd == 0.0) {   // zero reference: u = 0, projector = identity
+        r->cos = 0.0;
+        r->regime = GAC_REGIME_SAFE;
+        r->clip_scale = clip_factor(r->regime, dot, gg, dd, hp.beta, 0.0, hp.clip_max, hp.clip_eps, &r->out_norm);
+        return;
+    }
+    double c = __ddiv_rn(dot, __dadd_rn(__dsqrt_rn(__dmul_rn(gg, dd)), hp.eps));
+    double ac = fabs(c);
+    r->cos = c;
+    if (hp.mode == GAC_MODE_FIXED) {
+        r->regime = GAC_REGIME_PROJECT;
+        r->alpha = hp.alpha_fixed;
+    } else if (ac <= hp.c_low) {
+        r->regime = GAC_REGIME_SAFE;
+        r->clip_scale = clip_factor(r->regime, dot, gg, dd, hp.beta, 0.0, hp.clip_max, hp.clip_eps, &r->out_norm);
+        return;
+    } else if (ac >= hp.c_high) {
+        r->regime = GAC_REGIME_VIOLATION;
+        return;
+    } else {
+        r->regime = GAC_REGIME_PROJECT;
+        r->alpha = __ddiv_rn(hp.c_low, ac);
+    }
+    double k = __ddiv_rn(__dmul_rn(__dadd_rn(r->alpha, -hp.beta), dot), dd);
+    r->coef64 = k;
+    r->coef = __double2float_rn(k);
+    r->clip_scale = clip_factor(r->regime, dot, gg, dd, hp.beta, double(r->coef), hp.clip_max, hp.clip_eps,
+                                &r->out_norm);
+}
+
+// ------------------------------------------------------------- stats kernel
+
+__device__ __forceinline__ double warp_sum(double v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xFFFFFFFFu, v, o);
+    return v;
+}
+
+// Sums (a, b, c) over the CTA in a fixed order; the result is valid in thread 0.
+template <int T>
+__device__ __forceinline__ void block_sum3(double &a, double &b, double &c, double (*sm)[3]) {
+    a = warp_sum(a);
+    b = warp_sum(b);
+    c = warp_sum(c);
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    if (lane == 0) {
+        sm[warp][0] = a;
+        sm[warp][1] = b;
+        sm[warp][2] = c;
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        a = sm[0][0];
+        b = sm[0][1];
+        c = sm[0][2];
+        for (int w = 1; w < T / 32; ++w) {
+            a += sm[w][0];
+            b += sm[w][1];
+            c += sm[w][2];
+        }
+    }
+    __syncthreads();
+}
+
+template <typename GT, bool READ_D>
+__device__ __forceinline__ void stats_chunk(const Chunk &ch, double &a_dot, double &a_gg,
+                                            double &a_dd) {
+    const void *g = reinterpret_cast<const void *>(ch.g);
+    const void *d = reinterpret_cast<const void *>(ch.d);
+    const uint32_t tid = threadIdx.x;
+    constexpr int T = StatsGeom<GT>::T, U = StatsGeom<GT>::U;
+    if (ch.flags & kChunkAligned) {
+        const uint32_t nvec = ch.n >> 2;
+        for (uint32_t base = 0; base < nvec; base += T * U) {
+            F4 gv[U], dv[U];
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+                const uint32_t v = base + u * T + tid;
+                if (v < nvec) {
+                    gv[u] = Elem<GOf<GT>>::template load4<GAC_LD_STATS>(g, v);
+                    if (READ_D) dv[u] = Elem<DOf<GT>>::template load4<GAC_LD_STATS>(d, v);
+                } else {
+                    gv[u] = F4{0.f, 0.f, 0.f, 0.f};
+                    if (READ_D) dv[u] = F4{0.f, 0.f, 0.f, 0.f};
+                }
+            }
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+                const float ge[4] = {gv[u].x, gv[u].y, gv[u].z, gv[u].w};
+                const float de[4] = {dv[u].x, dv[u].y, dv[u].z, dv[u].w};
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    const double x = double(ge[e]);
+                    a_gg = fma(x, x, a_gg);
+                    if (READ_D) {
+                        const double y = double(de[e]);
+                        a_dot = fma(x, y, a_dot);
+                        a_dd = fma(y, y, a_dd);
+                    }
+                }
+            }
+        }
+        const uint32_t done = nvec << 2;
+        if (tid < ch.n - done) {   // ragged tail of a tensor: < 4 elements
+            const double x = double(Elem<GOf<GT>>::load1(g, done + tid));
+            a_gg = fma(x, x, a_gg);
+            if (READ_D) {
+                const double y = double(Elem<DOf<GT>>::load1(d, done + tid));
+                a_dot = fma(x, y, a_dot);
+                a_dd = fma(y, y, a_dd);
+            }
+        }
+    } else {   // a base that is not 16-byte aligned: element-wise, still coalesced
+        for (uint32_t i = tid; i < ch.n; i += T) {
+            const double x = double(Elem<GOf<GT>>::load1(g, i));
+            a_gg = fma(x, x, a_gg);
+            if (READ_D) {
+                const double y = double(Elem<DOf<GT>>::load1(d, i));
+                a_dot = fma(x, y, a_dot);
+                a_dd = fma(y, y, a_dd);
+            }
+        }
+    }
+}
+
+// partials: gridDim.x x 3 doubles, each slot written once per launch.
+// ticket: zero on entry; the last CTA to arrive reduces the slots in index
+// order, publishes the result and puts the ticket back to zero.  No CTA waits.
+template <typename GT>
+__global__ void __launch_bounds__(StatsGeom<GT>::T, StatsGeom<GT>::MINB)
+gac_stats_kernel(const Chunk *__restrict__ chunks, uint32_t n_chunks, double *partials,
+                 unsigned *ticket, gac_result *rec, double *sums_out, DevHP hp) {
+    constexpr int T = StatsGeom<GT>::T;
+    __shared__ double sm[T / 32][3];
+    __shared__ bool is_last;
+    double a_dot = 0.0, a_gg = 0.0, a_dd = 0.0;
+    if (hp.first_step) {
+        for (uint32_t c = blockIdx.x; c < n_chunks; c += gridDim.x)
+            stats_chunk<GT, false>(load_chunk(chunks, c), a_dot, a_gg, a_dd);
+    } else {
+        for (uint32_t c = blockIdx.x; c < n_chunks; c += gridDim.x)
+            stats_chunk<GT, true>(load_chunk(chunks, c), a_dot, a_gg, a_dd);
+    }
+    block_sum3<T>(a_dot, a_gg, a_dd, sm);
+    if (threadIdx.x == 0) {
+        double *slot = partials + 3 * size_t(blockIdx.x);
+        slot[0] = a_dot;
+        slot[1] = a_gg;
+        slot[2] = a_dd;
+        __threadfence();
+        const unsigned t = atomicAdd(ticket, 1u);
+        is_last = (t == gridDim.x - 1);
+    }
+    __syncthreads();
+    if (!is_last) return;
+    __threadfence();
+    // second stage: thread t adds slots t, t+T, t+2T, ... in that order, then the
+    // same fixed tree as above
+    double s0 = 0.0, s1 = 0.0, s2 = 0.0;
+    for (uint32_t b = threadIdx.x; b < gridDim.x; b += T) {
+        const double *slot = partials + 3 * size_t(b);
+        s0 += __ldcg(slot + 0);
+        s1 += __ldcg(slot + 1);
+        s2 += __ldcg(slot + 2);
+    }
+    block_sum3<T>(s0, s1, s2, sm);
+    if (threadIdx.x == 0) {
+        *ticket = 0u;
+        if (sums_out) {
+            sums_out[0] = hp.first_step ? 0.0 : s0;
+            sums_out[1] = s1;
+            sums_out[2] = hp.first_step ? 0.0 : s2;
+        }
+        if (hp.decide) take_decision(s0, s1, s2, hp, rec);
+    }
+}
+
+__global__ void gac_decide_kernel(const double *sums_in, gac_result *rec, DevHP hp) {
+    if (threadIdx.x == 0 && blockIdx.x == 0)
+        take_decision(sums_in[0], sums_in[1], sums_in[2], hp, rec);
+}
+
+// ----------------------------------------------------------- project kernel
+
+enum GOp { G_KEEP = 0, G_FMA = 1, G_ZERO = 2, G_SCALE = 3 };
+enum DOp { D_KEEP = 0, D_RAW = 1, D_NEW = 2 };
+
+template <bool BETA1>
+__device__ __forceinline__ float rank_one(float g, float d, float k, double beta, double s) {
+    if (BETA1) return fmaf(k, d, g);   // beta = 1, no clipping: one rounding
+    // general beta and/or an active clip factor s: binary64 (rounded product + exact product), times s
+    return __double2float_rn(
+        __dmul_rn(s, __dadd_rn(__dmul_rn(beta, double(g)), __dmul_rn(double(k), double(d)))));
+}
+__device__ __forceinline__ float scaled(float g, double s) { return __double2float_rn(__dmul_rn(s, double(g))); }
+
+template <typename GT, int GOP, int DOP, bool BETA1, int T, int U>
+__device__ __forceinline__ void project_chunk(const Chunk &ch, float k, double beta, double s) {
+    void *g = reinterpret_cast<void *>(ch.g);
+    void *d = reinterpret_cast<void *>(ch.d);
+    const uint32_t tid = threadIdx.x;
+    constexpr bool kReadG = (GOP == G_FMA) || (GOP == G_SCALE) || (DOP == D_RAW);
+    constexpr bool kReadD = (GOP == G_FMA);
+    if (ch.flags & kChunkAligned) {
+        const uint32_t nvec = ch.n >> 2;
+        for (uint32_t base = 0; base < nvec; base += T * U) {
+            F4 gv[U], dv[U];
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+                const uint32_t v = base + u * T + tid;
+                gv[u] = F4{0.f, 0.f, 0.f, 0.f};
+                dv[u] = F4{0.f, 0.f, 0.f, 0.f};
+                if (v < nvec) {
+                    if (kReadG) gv[u] = Elem<GOf<GT>>::template load4<GAC_LD_PROJECT>(g, v);
+                    if (kReadD) dv[u] = Elem<DOf<GT>>::template load4<GAC_LD_PROJECT>(d, v);
+                }
+            }
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+                const uint32_t v = base + u * T + tid;
+                if (v >= nvec) continue;
+                F4 out = gv[u];
+                if (GOP == G_ZERO) out = F4{0.f, 0.f, 0.f, 0.f};
+                if (GOP == G_FMA) {
+                    out.x = rank_one<BETA1>(gv[u].x, dv[u].x, k, beta, s);
+                    out.y = rank_one<BETA1>(gv[u].y, dv[u].y, k, beta, s);
+                    out.z = rank_one<BETA1>(gv[u].z, dv[u].z, k, beta, s);
+                    out.w = rank_one<BETA1>(gv[u].w, dv[u].w, k, beta, s);
+                }
+                if (GOP == G_SCALE) out = F4{scaled(gv[u].x, s), scaled(gv[u].y, s), scaled(gv[u].z, s), scaled(gv[u].w, s)};
+                if (GOP != G_KEEP) Elem<GOf<GT>>::store4(g, v, out);
+                if (DOP == D_RAW) Elem<DOf<GT>>::store4(d, v, gv[u]);
+                if (DOP == D_NEW) {
+                    if (GOP == G_FMA || GOP == G_SCALE) out = Elem<GOf<GT>>::template load4<GAC_LD_PROJECT>(g, v);   // the value as stored (rounded)
+                    Elem<DOf<GT>>::store4(d, v, out);
+                }
+            }
+        }
+        const uint32_t done = nvec << 2;
+        if (tid < ch.n - done) {
+            const uint32_t i = done + tid;
+            const float x = kReadG ? Elem<GOf<GT>>::load1(g, i) : 0.f;
+            float out = (GOP == G_ZERO) ? 0.f : x;
+            if (GOP == G_FMA) out = rank_one<BETA1>(x, Elem<DOf<GT>>::load1(d, i), k, beta, s);
+            if (GOP == G_SCALE) out = scaled(x, s);
+            if (GOP != G_KEEP) Elem<GOf<GT>>::store1(g, i, out);
+            if (DOP == D_RAW) Elem<DOf<GT>>::store1(d, i, x);
+            if (DOP == D_NEW) {
+                if (GOP == G_FMA || GOP == G_SCALE) out = Elem<GOf<GT>>::load1(g, i);
+                Elem<DOf<GT>>::store1(d, i, out);
+            }
+        }
+    } else {
+        for (uint32_t i = tid; i < ch.n; i += T) {
+            const float x = kReadG ? Elem<GOf<GT>>::load1(g, i) : 0.f;
+            float out = (GOP == G_ZERO) ? 0.f : x;
+            if (GOP == G_FMA) out = rank_one<BETA1>(x, Elem<DOf<GT>>::load1(d, i), k, beta, s);
+            if (GOP == G_SCALE) out = scaled(x, s);
+            if (GOP != G_KEEP) Elem<GOf<GT>>::store1(g, i, out);
+            if (DOP == D_RAW) Elem<DOf<GT>>::store1(d, i, x);
+            if (DOP == D_NEW) {
+                if (GOP == G_FMA || GOP == G_SCALE) out = Elem<GOf<GT>>::load1(g, i);
+                Elem<DOf<GT>>::store1(d, i, out);
+            }
+        }
+    }
+}
+
+template <typename GT, int GOP, int DOP, bool BETA1>
+__device__ __forceinline__ void project_walk(const Chunk *chunks, uint32_t n_chunks, float k,
+                                             double beta, double s) {
+    for (uint32_t c = blockIdx.x; c < n_chunks; c += gridDim.x)
+        project_chunk<GT, GOP, DOP, BETA1, ProjGeom<GT>::T, ProjGeom<GT>::U>(load_chunk(chunks, c), k, beta, s);
+}
+
+// The regime is read from the device-resident record, so no host round trip
+// separates the two passes; every CTA takes the same (uniform) branch.  What
+// the host already knows (state mode, beta == 1, zero_on_violation) is fixed at
+// compile time so that each instantiation holds only the loops it can reach.
+template <typename GT, int STATE, bool BETA1, bool ZERO>
+__global__ void __launch_bounds__(ProjGeom<GT>::T, ProjGeom<GT>::MINB)
+gac_project_kernel(const Chunk *__restrict__ chunks, uint32_t n_chunks, gac_result *rec,
+                   float coef_override, int use_override, double beta, double clip_max, double clip_eps) {
+    if (rec->nonfinite) return;   // reading taken for NaN/Inf: touch nothing
+    const int regime = rec->regime;
+    const float k = use_override ? coef_override : rec->coef;
+    constexpr int dop = STATE == GAC_STATE_RAW ? D_RAW : (STATE == GAC_STATE_PROJECTED ? D_NEW : D_KEEP);
+    double s = 1.0;
+    if (clip_max > 0.0) {
+        // recomputed here so that it belongs to the coefficient actually applied
+        double norm;
+        s = clip_factor(regime, rec->dot, rec->gg, rec->dd, beta, double(k), clip_max, clip_eps, &norm);
+        if (use_override && blockIdx.x == 0 && threadIdx.x == 0) {
+            rec->out_norm = norm;       // nobody reads these two fields during this launch
+            rec->clip_scale = s;
+        }
+    }
+    if (regime == GAC_REGIME_PROJECT) {
+        if (s != 1.0) project_walk<GT, G_FMA, dop, false>(chunks, n_chunks, k, beta, s);
+        else project_walk<GT, G_FMA, dop, BETA1>(chunks, n_chunks, k, beta, 1.0);
+    } else if (ZERO && regime == GAC_REGIME_VIOLATION) {
+        project_walk<GT, G_ZERO, dop, true>(chunks, n_chunks, k, 1.0, 1.0);
+    } else if (s != 1.0) {
+        project_walk<GT, G_SCALE, dop, true>(chunks, n_chunks, k, 1.0, s);   // safe step, clipped: g'' = s g
+    } else if (STATE != GAC_STATE_HOLD) {
+        project_walk<GT, G_KEEP, D_RAW, true>(chunks, n_chunks, k, 1.0, 1.0);   // d' = g, g untouched
+    }
+}
+
+// ------------------------------------------------ projection fused with AdamW
+
+struct __align__(16) OptChunk {
+    uint64_t p, m, v, pad;   // device addresses of the chunk's first parameter / moment elements
+};
+static_assert(sizeof(OptChunk) == 32, "optimizer chunk descriptors are read as two 16-byte words");
+
+struct AdamDev {
+    double lr, beta1, beta2, eps, weight_decay;
+};
+
+struct AdamConst {
+    double b1, c1, b2, c2;                       // moment recurrences
+    double step_size, inv_sqrt_bc2, eps, lr_wd;  // lr/(1-b1^t), 1/sqrt(1-b2^t), eps, lr*wd
+};
+
+// The outgoing gradient in binary64, unrounded: the moments are differences of
+// nearly equal terms often enough that a binary32 g' would cost them digits.
+template <int GOP>
+__device__ __forceinline__ double outgoing64(float g, float d, float k, double beta, double s) {
+    if (GOP == G_FMA)
+        return __dmul_rn(s, __dadd_rn(__dmul_rn(beta, double(g)), __dmul_rn(double(k), double(d))));
+    if (GOP == G_SCALE) return __dmul_rn(s, double(g));
+    return double(g);
+}
+
+// One element of: g' -> AdamW, in binary64 so that p - delta stays accurate
+// even where it cancels (tiny parameters).  The square root and the reciprocal
+// start from binary32 hardware results and take one Newton step each in
+// binary64 (relative error ~1e-14), far cheaper than the binary64 library
+// routines.  m, v and p are each rounded once on the way out.
+__device__ __forceinline__ void adamw_elem(double g64, float &p, float &m, float &v, const AdamConst &a) {
+    const double m64 = __dadd_rn(__dmul_rn(a.b1, double(m)), __dmul_rn(a.c1, g64));
+    const double v64 = __dadd_rn(__dmul_rn(a.b2, double(v)), __dmul_rn(__dmul_rn(a.c2, g64), g64));
+    double root = 0.0;
+    const float r32 = __fsqrt_rn(__double2float_rn(v64));
+    if (r32 > 0.0f) {
+        const double r = double(r32);
+        root = fma(fma(-r, r, v64), double(__fdividef(0.5f, r32)), r);   // r + (v - r^2)/(2r)
+    }
+    const double denom = fma(root, a.inv_sqrt_bc2, a.eps);
+    const double q = double(__frcp_rn(__double2float_rn(denom)));
+    const double inv = q * fma(-denom, q, 2.0);                           // q (2 - denom q)
+    const double delta = fma(a.lr_wd, double(p), a.step_size * (m64 * inv));
+    p = __double2float_rn(double(p) - delta);
+    m = __double2float_rn(m64);
+    v = __double2float_rn(v64);
+}
+
+template <typename GT, int GOP>
+__device__ __forceinline__ void adamw_chunk(const Chunk &ch, const OptChunk &oc, float k, double beta,
+                                            double s, const AdamConst &a) {
+    const void *g = reinterpret_cast<const void *>(ch.g);
+    void *d = reinterpret_cast<void *>(ch.d);
+    void *pp = reinterpret_cast<void *>(oc.p);
+    void *pm = reinterpret_cast<void *>(oc.m);
+    void *pv = reinterpret_cast<void *>(oc.v);
+    const uint32_t tid = threadIdx.x;
+    constexpr int T = AdamGeom<GT>::T, U = AdamGeom<GT>::U;
+    const bool vec = (ch.flags & kChunkAligned) && ((oc.p | oc.m | oc.v) % 16 == 0);
+    if (vec) {
+        const uint32_t nvec = ch.n >> 2;
+        for (uint32_t base = 0; base < nvec; base += T * U) {
+            F4 gv[U], dv[U], p4[U], m4[U], v4[U];
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+                const uint32_t w = base + u * T + tid;
+                dv[u] = F4{0.f, 0.f, 0.f, 0.f};
+                if (w < nvec) {
+                    gv[u] = Elem<GOf<GT>>::template load4<GAC_LD_PROJECT>(g, w);
+                    if (GOP == G_FMA) dv[u] = Elem<DOf<GT>>::template load4<GAC_LD_PROJECT>(d, w);
+                    p4[u] = Elem<float>::load4<GAC_LD_PROJECT>(pp, w);
+                    m4[u] = Elem<float>::load4<GAC_LD_PROJECT>(pm, w);
+                    v4[u] = Elem<float>::load4<GAC_LD_PROJECT>(pv, w);
+                }
+            }
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+                const uint32_t w = base + u * T + tid;
+                if (w >= nvec) continue;
+                float ge[4] = {gv[u].x, gv[u].y, gv[u].z, gv[u].w};
+                float pe[4] = {p4[u].x, p4[u].y, p4[u].z, p4[u].w};
+                float me[4] = {m4[u].x, m4[u].y, m4[u].z, m4[u].w};
+                float ve[4] = {v4[u].x, v4[u].y, v4[u].z, v4[u].w};
+                const float de[4] = {dv[u].x, dv[u].y, dv[u].z, dv[u].w};
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    adamw_elem(outgoing64<GOP>(ge[e], de[e], k, beta, s), pe[e], me[e], ve[e], a);
+                }
+                Elem<DOf<GT>>::store4(d, w, gv[u]);                       // d' = g, the raw gradient
+                Elem<float>::store4(pp, w, F4{pe[0], pe[1], pe[2], pe[3]});
+                Elem<float>::store4(pm, w, F4{me[0], me[1], me[2], me[3]});
+                Elem<float>::store4(pv, w, F4{ve[0], ve[1], ve[2], ve[3]});
+            }
+        }
+    }
+    const uint32_t first = vec ? ((ch.n >> 2) << 2) : 0u;
+    for (uint32_t i = first + tid; i < ch.n; i += T) {
+        const float x = Elem<GOf<GT>>::load1(g, i);
+        const float dx = (GOP == G_FMA) ? Elem<DOf<GT>>::load1(d, i) : 0.f;
+        float pe = Elem<float>::load1(pp, i), me = Elem<float>::load1(pm, i), ve = Elem<float>::load1(pv, i);
+        adamw_elem(outgoing64<GOP>(x, dx, k, beta, s), pe, me, ve, a);
+        Elem<DOf<GT>>::store1(d, i, x);
+        Elem<float>::store1(pp, i, pe);
+        Elem<float>::store1(pm, i, me);
+        Elem<float>::store1(pv, i, ve);
+    }
+}
+
+__device__ __forceinline__ OptChunk load_opt_chunk(const OptChunk *table, uint32_t c) {
+    const uint4 *q = reinterpret_cast<const uint4 *>(table + c);
+    uint4 a = __ldg(q), b = __ldg(q + 1);
+    OptChunk oc;
+    oc.p = (uint64_t(a.y) << 32) | a.x;
+    oc.m = (uint64_t(a.w) << 32) | a.z;
+    oc.v = (uint64_t(b.y) << 32) | b.x;
+    oc.pad = 0;
+    return oc;
+}
+
+// Same decision logic as gac_project_kernel; a safe or projection step feeds
+// AdamW, a violation step only refreshes the stored direction.  The count of
+// applied updates lives in the decision record: every CTA reads it on entry,
+// and the last CTA to FINISH (arrival ticket, nobody waits) writes it back
+// incremented, so no CTA can see the new value during this launch.
+template <typename GT>
+__global__ void __launch_bounds__(AdamGeom<GT>::T, AdamGeom<GT>::C)
+gac_adamw_kernel(const Chunk *__restrict__ chunks, const OptChunk *__restrict__ opt_chunks,
+                 uint32_t n_chunks, gac_result *rec, unsigned *ticket, float coef_override,
+                 int use_override, double beta, double clip_max, double clip_eps, AdamDev o) {
+    if (rec->nonfinite) return;
+    const int regime = rec->regime;
+    const float k = use_override ? coef_override : rec->coef;
+    const unsigned long long t_prev = rec->applied_steps;
+    double s = 1.0;
+    if (clip_max > 0.0) {
+        double norm;
+        s = clip_factor(regime, rec->dot, rec->gg, rec->dd, beta, double(k), clip_max, clip_eps, &norm);
+        if (use_override && blockIdx.x == 0 && threadIdx.x == 0) {
+            rec->out_norm = norm;
+            rec->clip_scale = s;
+        }
+    }
+    const bool applies = (regime != GAC_REGIME_VIOLATION);
+    if (applies) {
+        const double t = double(t_prev + 1ull);
+        const double bc1 = 1.0 - pow(o.beta1, t), bc2 = 1.0 - pow(o.beta2, t);
+        AdamConst a;
+        a.b1 = o.beta1;
+        a.c1 = 1.0 - o.beta1;
+        a.b2 = o.beta2;
+        a.c2 = 1.0 - o.beta2;
+        a.step_size = o.lr / bc1;
+        a.inv_sqrt_bc2 = 1.0 / sqrt(bc2);
+        a.eps = o.eps;
+        a.lr_wd = o.lr * o.weight_decay;
+        for (uint32_t c = blockIdx.x; c < n_chunks; c += gridDim.x) {
+            const Chunk ch = load_chunk(chunks, c);
+            const OptChunk oc = load_opt_chunk(opt_chunks, c);
+            if (regime == GAC_REGIME_PROJECT) adamw_chunk<GT, G_FMA>(ch, oc, k, beta, s, a);
+            else if (s != 1.0) adamw_chunk<GT, G_SCALE>(ch, oc, k, 1.0, s, a);
+            else adamw_chunk<GT, G_KEEP>(ch, oc, k, 1.0, 1.0, a);
+        }
+    } else {
+        for (uint32_t c = blockIdx.x; c < n_chunks; c += gridDim.x)   // skipped step: d' = g only
+            project_chunk<GT, G_KEEP, D_RAW, true, AdamGeom<GT>::T, AdamGeom<GT>::U>(load_chunk(chunks, c), k, 1.0, 1.0);
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        __threadfence();
+        const unsigned done = atomicAdd(ticket, 1u);
+        if (done == gridDim.x - 1) {
+            rec->applied_steps = t_prev + (applies ? 1ull : 0ull);
+            __threadfence();
+            *ticket = 0u;
+        }
+    }
+}
+
+using ProjectKernel = void (*)(const Chunk *, uint32_t, gac_result *, float, int, double, double, double);
+
+template <typename GT, int STATE>
+ProjectKernel pick_project(bool beta1, bool zero) {
+    if (beta1) return zero ? gac_project_kernel<GT, STATE, true, true> : gac_project_kernel<GT, STATE, true, false>;
+    return zero ? gac_project_kernel<GT, STATE, false, true> : gac_project_kernel<GT, STATE, false, false>;
+}
+template <typename GT>
+ProjectKernel pick_project(int state, bool beta1, bool zero) {
+    if (state == GAC_STATE_RAW) return pick_project<GT, GAC_STATE_RAW>(beta1, zero);
+    if (state == GAC_STATE_PROJECTED) return pick_project<GT, GAC_STATE_PROJECTED>(beta1, zero);
+    return pick_project<GT, GAC_STATE_HOLD>(beta1, zero);
+}
+
+}  // namespace

@@ -98,6 +98,10 @@ def test_argument_errors_need_no_device(lib):
     assert _init(lib, [(4097, 8192, 16)])[0] == gb.GAC_ERR_INVALID_ARG       # not element-aligned
     rc, msg = _init(lib, [(4096, 4100, 16)])                                   # g and d overlap
     assert rc == gb.GAC_ERR_INVALID_ARG and "overlap" in msg
+    rc, msg = _init(lib, [(4096, 8192, 16), (16384, 4096 + 32, 16)])          # d of tensor 1 inside g of tensor 0
+    assert rc == gb.GAC_ERR_INVALID_ARG and "overlap" in msg
+    assert _init(lib, [ok], clip_max_norm=-1.0)[0] == gb.GAC_ERR_INVALID_ARG
+    assert _init(lib, [ok], g_dt=1, d_dt=1)[0] in (gb.GAC_OK, gb.GAC_ERR_CUDA)   # bf16/bf16 is a supported pair
     rc, msg = _init(lib, [ok])
     # with valid arguments the only thing that can fail here is the missing device
     import torch

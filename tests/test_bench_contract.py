@@ -1,0 +1,46 @@
+"""bench.py prints one JSON line with the agreed keys (reference arm on CPU;
+the library's arm on a GPU, on a small list so that it ends in seconds)."""
+import json
+import os
+import subprocess
+import sys
+
+import pytest
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+BASE = {"metric", "value", "unit", "n_gpus", "steps", "warmup", "ms_per_step", "higher_is_better",
+        "scaling", "vs_baseline", "dtype", "data", "config", "e2e"}
+
+
+def run_bench(*args):
+    out = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), *args], capture_output=True,
+                         text=True, timeout=900, cwd=ROOT)
+    assert out.returncode == 0, out.stderr[-2000:]
+    lines = [l for l in out.stdout.splitlines() if l.startswith("{")]
+    assert len(lines) == 1, out.stdout[-2000:]
+    return json.loads(lines[0])
+
+
+def test_reference_arm_runs_the_oracle_on_the_host():
+    d = run_bench("--impl", "reference", "--workload", "small_f32", "--steps", "2", "--warmup", "3")
+    assert BASE <= set(d)
+    assert d["impl"] == "reference" and d["unit"] == "params/s" and d["value"] > 0
+    assert d["cpu_baseline"]["kind"] == "oracle" and d["cpu_baseline"]["cores"] >= 1
+    assert d["e2e"]["h2d_bytes_per_step"] == 0 and d["e2e"]["d2h_bytes_per_step"] == 0
+    assert "workload" in d["config"] and "model" not in d["config"]
+
+
+@pytest.mark.gpu
+def test_library_arm_line_on_a_small_list():
+    d = run_bench("--workload", "small_bf16", "--also", "small_f32", "--steps", "3", "--warmup", "3")
+    assert BASE <= set(d)
+    assert d["n_gpus"] == 1 and d["data"] == "synthetic" and d["vs_baseline"] is None
+    assert d["gpu_launches"] == 2 * d["steps"]
+    r = d["roofline"]
+    assert r["bound"] == "hbm" and r["unit"] == "GB/s" and abs(r["frac"] - r["achieved"] / r["peak"]) < 1e-9
+    assert d["regime_check"]["regime"] == "project" and abs(d["regime_check"]["cos"] - 0.95) < 0.01
+    assert d["e2e"]["h2d_bytes_per_step"] > 0 and d["e2e"]["d2h_bytes_per_step"] > d["e2e"]["h2d_bytes_per_step"]
+    assert d["cpu_baseline"]["kind"] == "oracle"
+    assert {"sm_mhz", "sm_max_mhz", "reasons"} <= set(d["clocks"])
+    assert d["also"]["regime_check"]["regime"] == "project"
+    assert d["unchanged_regime"]["regime"] == "violation"
