@@ -94,6 +94,17 @@ namespace {
 #ifndef GAC_PROJ_MINB_BF16X
 #define GAC_PROJ_MINB_BF16X GAC_PROJ_MINB_BF16
 #endif
+// vectors in flight per thread when a step leaves g alone (safe / violation): only g is
+// read and only d written, so each vector carries fewer bytes than in the projection
+#ifndef GAC_KEEP_U_F32
+#define GAC_KEEP_U_F32 16
+#endif
+#ifndef GAC_KEEP_U_BF16
+#define GAC_KEEP_U_BF16 8
+#endif
+#ifndef GAC_KEEP_U_BF16X
+#define GAC_KEEP_U_BF16X 8
+#endif
 #ifndef GAC_ADAMW_T_F32
 #define GAC_ADAMW_T_F32 1024
 #endif
@@ -247,14 +258,17 @@ template <typename GT>
 struct ProjGeom;
 template <>
 struct ProjGeom<float> {
+    static constexpr int UK = GAC_KEEP_U_F32;
     static constexpr int T = GAC_PROJ_T_F32, U = GAC_PROJ_U_F32, C = GAC_PROJ_C_F32, MINB = GAC_PROJ_MINB_F32;
 };
 template <>
 struct ProjGeom<bf16_t> {
+    static constexpr int UK = GAC_KEEP_U_BF16;
     static constexpr int T = GAC_PROJ_T_BF16, U = GAC_PROJ_U_BF16, C = GAC_PROJ_C_BF16, MINB = GAC_PROJ_MINB_BF16;
 };
 template <>
 struct ProjGeom<bf16_pair_t> {
+    static constexpr int UK = GAC_KEEP_U_BF16X;
     static constexpr int T = GAC_PROJ_T_BF16X, U = GAC_PROJ_U_BF16X, C = GAC_PROJ_C_BF16X, MINB = GAC_PROJ_MINB_BF16X;
 };
 
@@ -647,7 +661,8 @@ gac_project_kernel(const Chunk *__restrict__ chunks, uint32_t n_chunks, gac_resu
     } else if (s != 1.0) {
         project_walk<GT, G_SCALE, dop, true>(chunks, n_chunks, k, 1.0, s);   // safe step, clipped: g'' = s g
     } else if (STATE != GAC_STATE_HOLD) {
-        project_walk<GT, G_KEEP, D_RAW, true>(chunks, n_chunks, k, 1.0, 1.0);   // d' = g, g untouched
+        for (uint32_t c = blockIdx.x; c < n_chunks; c += gridDim.x)   // d' = g, g untouched
+            project_chunk<GT, G_KEEP, D_RAW, true, ProjGeom<GT>::T, ProjGeom<GT>::UK>(load_chunk(chunks, c), k, 1.0, 1.0);
     }
 }
 
