@@ -141,7 +141,7 @@ def recorded_traffic(kernel: str):
 # --------------------------------------------------------------- GPU workload
 
 class Workload:
-    def __init__(self, name: str, device, world: int, clip: float = 0.0):
+    def __init__(self, name: str, device, world: int, clip: float = 0.0, sharded: bool = False):
         from paper_2603_01501_b200 import binding as gb
         self.gb = gb
         dims_key, self.g_dtype, self.rho, self.config_id = synth.WORKLOADS[name]
@@ -158,7 +158,8 @@ class Workload:
         self.gen.manual_seed(12345 + self.config_id)
         self.ctx = gb.gac_init(self.g, self.d, gb.HParams(clip_max_norm=clip, **FORCE))
         self.step_no = 1      # the stored direction already holds g_{t-1}
-        self.sums = torch.zeros(3, dtype=torch.float64, device=device) if world > 1 else None
+        self.sharded = sharded or world > 1     # local sums -> all-reduce -> decision (App. A.1)
+        self.sums = torch.zeros(3, dtype=torch.float64, device=device) if self.sharded else None
 
     def refresh(self):
         synth.refresh_gradient_list(self.g, self.d, self.sigma, self.rho, self.gen, self.scratch)
@@ -169,7 +170,7 @@ class Workload:
         self.step_no += 1
         if ev:
             ev[0].record()
-        if self.world > 1:
+        if self.sharded:
             # sharded form (App. A.1): local sums, ONE all-reduce of three numbers, same decision on every rank
             gb.gac_stats_partial(self.ctx, self.step_no, self.sums)
             torch.distributed.all_reduce(self.sums)
@@ -300,7 +301,7 @@ def check_regime(wl: Workload):
     wl.refresh()
     gb = wl.gb
     wl.step_no += 1
-    if wl.world > 1:
+    if wl.sharded:
         gb.gac_stats_partial(wl.ctx, wl.step_no, wl.sums)
         torch.distributed.all_reduce(wl.sums)
         res = gb.gac_decide(wl.ctx, wl.sums)
@@ -483,6 +484,9 @@ def main():
                     help="second workload reported under 'also' (1 GPU only); 'none' to skip")
     ap.add_argument("--clip", type=float, default=0.0,
                     help="fold global-norm clipping with this max norm into the projection pass (0 = off)")
+    ap.add_argument("--sharded", action="store_true",
+                    help="use the sharded call sequence (local sums, NCCL all-reduce of 3 doubles, decision) "
+                         "even on one GPU; always on for --gpus > 1")
     ap.add_argument("--adamw", action="store_true",
                     help="also time the projection fused with AdamW on the main workload (1 GPU)")
     ap.add_argument("--no-e2e", action="store_true")
@@ -504,12 +508,13 @@ def main():
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
     torch.cuda.set_device(local_rank)
     device = torch.device("cuda", local_rank)
-    if world > 1:
+    if world > 1 or args.sharded:
         os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
-        torch.distributed.init_process_group("nccl", device_id=device)
+        os.environ.setdefault("MASTER_PORT", "29577")
+        torch.distributed.init_process_group("nccl", device_id=device, rank=rank, world_size=world)
     peak, peak_kind = measured_hbm_peak()
 
-    wl = Workload(args.workload, device, world, args.clip)
+    wl = Workload(args.workload, device, world, args.clip, args.sharded)
     sampler = ClockSampler(nvml_index(local_rank))
     wall0 = time.perf_counter()
     s_ms, p_ms = time_steps(wl, args.steps, args.warmup, sampler)
@@ -534,7 +539,7 @@ def main():
                              "clip_scale": res.clip_scale},
             "launch": {"grid": info.grid, "threads": info.threads, "chunk_elems": info.chunk_elems,
                        "chunks": info.n_chunks},
-            "gpu_launches": (2 if world == 1 else 3) * args.steps,
+            "gpu_launches": (3 if wl.sharded else 2) * args.steps,
             "clocks": sampler.summary(), "roofline": summ["roofline"],
             "roofline_stats": summ["roofline_stats"], "wall_s_timed_loop": wall}
     if world > 1:
@@ -597,7 +602,7 @@ def main():
         cb = time_oracle(args.workload, target, passes, 0)
         line["cpu_baseline"] = {k: cb[k] for k in ("value", "unit", "cores", "kind", "sample")}
 
-    if world > 1:
+    if world > 1 or args.sharded:
         torch.distributed.barrier()
         torch.distributed.destroy_process_group()
     if rank == 0:

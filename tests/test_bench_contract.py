@@ -44,3 +44,13 @@ def test_library_arm_line_on_a_small_list():
     assert {"sm_mhz", "sm_max_mhz", "reasons"} <= set(d["clocks"])
     assert d["also"]["regime_check"]["regime"] == "project"
     assert d["unchanged_regime"]["regime"] == "violation"
+
+
+@pytest.mark.gpu
+def test_sharded_call_sequence_with_a_one_rank_nccl_group():
+    """The multi-GPU call sequence (local sums, NCCL all-reduce of three doubles, decision,
+    projection) on one GPU: same numbers as the unsharded line, three launches per step."""
+    d = run_bench("--workload", "small_f32", "--also", "none", "--steps", "3", "--warmup", "3", "--sharded",
+                  "--no-e2e", "--no-cpu-baseline")
+    assert d["gpu_launches"] == 3 * d["steps"]
+    assert d["regime_check"]["regime"] == "project" and abs(d["regime_check"]["cos"] - 0.9) < 0.01

@@ -1,5 +1,5 @@
 """Pins the CPU oracle to what the paper and mathematics fix, before it is
-trusted as the judge of the CUDA library.  Nothing here touches a GPU.
+trusted as the arbiter of the CUDA library.  Nothing here touches a GPU.
 
 Each test is chosen so that one plausible mistake in the oracle (a dropped
 term, a wrong sign, eps in the wrong place, an exclusive threshold, a
