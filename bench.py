@@ -459,6 +459,7 @@ def summarize(wl: Workload, s_ms, p_ms, peak, peak_kind):
     return {
         "ms_per_step": step_ms, "stats_ms": s_avg, "project_ms": p_avg,
         "best_ms_per_step": min(a + b for a, b in zip(s_ms, p_ms)),
+        "median_ms_per_step": statistics.median(a + b for a, b in zip(s_ms, p_ms)),
         "hbm_gbs": (proj_bytes + stats_bytes) / (step_ms * 1e-3) / 1e9,
         "roofline": {"bound": "hbm", "kernel": "gac_project_kernel", "achieved": proj_gbs,
                      "peak": peak, "unit": "GB/s", "frac": proj_gbs / peak,
@@ -535,6 +536,7 @@ def main():
             "hbm_gbs": summ["hbm_gbs"] , "frac_of_nominal_8TBs": summ["hbm_gbs"] / NOMINAL_HBM_GBS,
             "stats_ms": summ["stats_ms"], "project_ms": summ["project_ms"],
             "best_ms_per_step": summ["best_ms_per_step"],
+            "median_ms_per_step": summ["median_ms_per_step"],
             "regime_check": {"cos": res.cos, "regime": gb.REGIME_NAMES[res.regime], "alpha": res.alpha,
                              "clip_scale": res.clip_scale},
             "launch": {"grid": info.grid, "threads": info.threads, "chunk_elems": info.chunk_elems,

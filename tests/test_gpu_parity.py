@@ -377,3 +377,71 @@ def test_step_can_be_captured_in_a_cuda_graph_and_replayed():
         assert max_ulp(g[0].cpu(), g_ref[0]) <= 64      # own coefficient: may differ in its last bit
         assert float((g[0].cpu().double() - g_ref[0].double()).abs().max()) <= 2e-7 * float(g_new.abs().max())
     gb.gac_free(ctx)
+
+
+@pytest.mark.parametrize("seed", range(12))
+def test_random_list_structures(seed):
+    """Random lists: tiny and large tensors mixed, some as odd-offset views, random element types,
+    thresholds and chunk sizes -- the chunk table must present them all as one flat vector."""
+    import random
+    rng = random.Random(seed)
+    g_dtype = rng.choice([torch.float32, torch.bfloat16])
+    n_t = rng.randint(1, 40)
+    sizes = [rng.choice([1, 2, 3, 5, 17, 255, 1024, 4097, 16384, 16385, 70001, rng.randint(1, 300000)])
+             for _ in range(n_t)]
+    rho = rng.choice([0.0, 0.1, 0.5, 0.95, -0.7])
+    gen = torch.Generator().manual_seed(seed)
+    g_cpu, d_cpu, g_gpu, d_gpu = [], [], [], []
+    for n in sizes:
+        scale = 10.0 ** rng.uniform(-4, 0)
+        d = torch.randn(n, generator=gen) * scale
+        g = (rho * d + math.sqrt(1 - rho * rho) * torch.randn(n, generator=gen) * scale).to(g_dtype)
+        g_cpu.append(g)
+        d_cpu.append(d)
+        og, od = (rng.randint(0, 7), rng.randint(0, 7)) if rng.random() < 0.3 else (0, 0)
+        gbuf = torch.zeros(n + 8, dtype=g_dtype, device="cuda")
+        dbuf = torch.zeros(n + 8, dtype=torch.float32, device="cuda")
+        gbuf[og:og + n] = g.cuda()
+        dbuf[od:od + n] = d.cuda()
+        g_gpu.append(gbuf[og:og + n])
+        d_gpu.append(dbuf[od:od + n])
+    hp = rng.choice([gb.HParams(), gb.HParams(**FORCE), gb.HParams(c_low=0.3, c_high=0.6),
+                     gb.HParams(mode=gb.GAC_MODE_FIXED, alpha_fixed=0.0),
+                     gb.HParams(**FORCE, clip_max_norm=0.5)])
+    ohp = to_orc_hp(hp)
+    g_ref, d_ref = [t.clone() for t in g_cpu], [t.clone() for t in d_cpu]
+    dec = orc.step(g_ref, d_ref, ohp)
+    ctx = gb.gac_init(g_gpu, d_gpu, hp)
+    gb.gac_set_launch(ctx, rng.choice([1024, 4096, 16384, 32768]), rng.choice([0, 1, 3]))
+    res = gb.gac_stats(ctx, 2)
+    gb.gac_project(ctx, coef_override=dec.coef if dec.regime == orc.PROJECT else None)
+    torch.cuda.synchronize()
+    gb.gac_free(ctx)
+    check_sums(res, dec)
+    if abs(abs(dec.cos) - hp.c_low) > 1e-4 and abs(abs(dec.cos) - hp.c_high) > 1e-4:
+        check_decision(res, dec)
+        check_outputs(g_gpu, d_gpu, g_ref, d_ref)
+
+
+def test_state_recurrence_is_bitwise_and_survives_a_new_context():
+    """With the raw gradient as state, <d,d> of step t+1 is <g,g> of step t bit for bit (same values
+    summed in the same order), also when step t+1 runs in a fresh context on the same buffers."""
+    shapes = synth.decoder_tensor_list(synth.DIMS["small"])
+    for g_dtype in (torch.float32, torch.bfloat16):
+        g, d = synth.gradient_list(shapes, 0.3, config_id=2, g_dtype=g_dtype, device="cuda")
+        hp = gb.HParams(**FORCE)
+        ctx = gb.gac_init(g, d, hp)
+        r1 = gb.gac_stats(ctx, 5)
+        gb.gac_project(ctx)
+        for t in g:
+            t.copy_((torch.randn(t.numel(), device="cuda") * 0.01).to(g_dtype))
+        r2 = gb.gac_stats(ctx, 6)
+        assert r2.dd == r1.gg
+        gb.gac_project(ctx)
+        gb.gac_free(ctx)
+        ctx = gb.gac_init(g, d, hp)            # resume: same buffers, later step
+        for t in g:
+            t.copy_((torch.randn(t.numel(), device="cuda") * 0.01).to(g_dtype))
+        r3 = gb.gac_stats(ctx, 7)
+        assert r3.dd == r2.gg and r3.step == 7
+        gb.gac_free(ctx)
