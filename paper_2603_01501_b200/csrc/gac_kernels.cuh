@@ -13,116 +13,6 @@
 
 namespace {
 
-// Launch geometry.  Both kernels are bound by HBM, and on B200 their speed
-// depends on how many bytes each SM keeps in flight: too few starve the
-// memory system, too many make reads and write-backs of many chunks collide in
-// DRAM.  The macros exist so that variants can be built and timed side by side;
-// the defaults are the measured best per element type (T threads per CTA,
-// U four-element vectors in flight per thread and operand, C resident CTAs per
-// SM the grid is sized for with 0 = all that fit, MINB = occupancy asked of the
-// compiler with 0 = no request).
-#ifndef GAC_STATS_T_F32
-#define GAC_STATS_T_F32 256
-#endif
-#ifndef GAC_STATS_U_F32
-#define GAC_STATS_U_F32 8
-#endif
-#ifndef GAC_STATS_C_F32
-#define GAC_STATS_C_F32 0
-#endif
-#ifndef GAC_STATS_MINB_F32
-#define GAC_STATS_MINB_F32 4
-#endif
-#ifndef GAC_STATS_T_BF16
-#define GAC_STATS_T_BF16 256
-#endif
-#ifndef GAC_STATS_U_BF16
-#define GAC_STATS_U_BF16 8
-#endif
-#ifndef GAC_STATS_C_BF16
-#define GAC_STATS_C_BF16 0
-#endif
-#ifndef GAC_STATS_MINB_BF16
-#define GAC_STATS_MINB_BF16 4
-#endif
-#ifndef GAC_PROJ_T_F32
-#define GAC_PROJ_T_F32 256
-#endif
-#ifndef GAC_PROJ_U_F32
-#define GAC_PROJ_U_F32 8
-#endif
-#ifndef GAC_PROJ_C_F32
-#define GAC_PROJ_C_F32 1
-#endif
-#ifndef GAC_PROJ_MINB_F32
-#define GAC_PROJ_MINB_F32 1
-#endif
-#ifndef GAC_PROJ_T_BF16
-#define GAC_PROJ_T_BF16 512
-#endif
-#ifndef GAC_PROJ_U_BF16
-#define GAC_PROJ_U_BF16 4
-#endif
-#ifndef GAC_PROJ_C_BF16
-#define GAC_PROJ_C_BF16 1
-#endif
-#ifndef GAC_PROJ_MINB_BF16
-#define GAC_PROJ_MINB_BF16 1
-#endif
-// (bfloat16 g, bfloat16 d): half the bytes per vector of the mixed pair
-#ifndef GAC_STATS_T_BF16X
-#define GAC_STATS_T_BF16X GAC_STATS_T_BF16
-#endif
-#ifndef GAC_STATS_U_BF16X
-#define GAC_STATS_U_BF16X GAC_STATS_U_BF16
-#endif
-#ifndef GAC_STATS_C_BF16X
-#define GAC_STATS_C_BF16X GAC_STATS_C_BF16
-#endif
-#ifndef GAC_STATS_MINB_BF16X
-#define GAC_STATS_MINB_BF16X GAC_STATS_MINB_BF16
-#endif
-#ifndef GAC_PROJ_T_BF16X
-#define GAC_PROJ_T_BF16X GAC_PROJ_T_BF16
-#endif
-#ifndef GAC_PROJ_U_BF16X
-#define GAC_PROJ_U_BF16X 8
-#endif
-#ifndef GAC_PROJ_C_BF16X
-#define GAC_PROJ_C_BF16X GAC_PROJ_C_BF16
-#endif
-#ifndef GAC_PROJ_MINB_BF16X
-#define GAC_PROJ_MINB_BF16X GAC_PROJ_MINB_BF16
-#endif
-// vectors in flight per thread when a step leaves g alone (safe / violation): only g is
-// read and only d written, so each vector carries fewer bytes than in the projection
-#ifndef GAC_KEEP_U_F32
-#define GAC_KEEP_U_F32 16
-#endif
-#ifndef GAC_KEEP_U_BF16
-#define GAC_KEEP_U_BF16 8
-#endif
-#ifndef GAC_KEEP_U_BF16X
-#define GAC_KEEP_U_BF16X 8
-#endif
-#ifndef GAC_ADAMW_T_F32
-#define GAC_ADAMW_T_F32 1024
-#endif
-#ifndef GAC_ADAMW_U_F32
-#define GAC_ADAMW_U_F32 1
-#endif
-#ifndef GAC_ADAMW_C_F32
-#define GAC_ADAMW_C_F32 1
-#endif
-#ifndef GAC_ADAMW_T_BF16
-#define GAC_ADAMW_T_BF16 1024
-#endif
-#ifndef GAC_ADAMW_U_BF16
-#define GAC_ADAMW_U_BF16 1
-#endif
-#ifndef GAC_ADAMW_C_BF16
-#define GAC_ADAMW_C_BF16 1
-#endif
 #ifndef GAC_CHUNK
 #define GAC_CHUNK 16384
 #endif
@@ -228,49 +118,37 @@ using GOf = typename PairOf<P>::G;
 template <typename P>
 using DOf = typename PairOf<P>::D;
 
-template <typename GT>
-struct StatsGeom;
-template <>
-struct StatsGeom<float> {
-    static constexpr int T = GAC_STATS_T_F32, U = GAC_STATS_U_F32, C = GAC_STATS_C_F32, MINB = GAC_STATS_MINB_F32;
-};
-template <>
-struct StatsGeom<bf16_t> {
-    static constexpr int T = GAC_STATS_T_BF16, U = GAC_STATS_U_BF16, C = GAC_STATS_C_BF16, MINB = GAC_STATS_MINB_BF16;
-};
-template <typename GT>
-struct AdamGeom;
-template <>
-struct AdamGeom<float> {
-    static constexpr int T = GAC_ADAMW_T_F32, U = GAC_ADAMW_U_F32, C = GAC_ADAMW_C_F32;
-};
-template <>
-struct AdamGeom<bf16_t> {
-    static constexpr int T = GAC_ADAMW_T_BF16, U = GAC_ADAMW_U_BF16, C = GAC_ADAMW_C_BF16;
-};
-template <>
-struct StatsGeom<bf16_pair_t> {
-    static constexpr int T = GAC_STATS_T_BF16X, U = GAC_STATS_U_BF16X, C = GAC_STATS_C_BF16X, MINB = GAC_STATS_MINB_BF16X;
-};
-template <>
-struct AdamGeom<bf16_pair_t> : AdamGeom<bf16_t> {};
-template <typename GT>
-struct ProjGeom;
-template <>
-struct ProjGeom<float> {
-    static constexpr int UK = GAC_KEEP_U_F32;
-    static constexpr int T = GAC_PROJ_T_F32, U = GAC_PROJ_U_F32, C = GAC_PROJ_C_F32, MINB = GAC_PROJ_MINB_F32;
-};
-template <>
-struct ProjGeom<bf16_t> {
-    static constexpr int UK = GAC_KEEP_U_BF16;
-    static constexpr int T = GAC_PROJ_T_BF16, U = GAC_PROJ_U_BF16, C = GAC_PROJ_C_BF16, MINB = GAC_PROJ_MINB_BF16;
-};
-template <>
-struct ProjGeom<bf16_pair_t> {
-    static constexpr int UK = GAC_KEEP_U_BF16X;
-    static constexpr int T = GAC_PROJ_T_BF16X, U = GAC_PROJ_U_BF16X, C = GAC_PROJ_C_BF16X, MINB = GAC_PROJ_MINB_BF16X;
-};
+// Launch geometry.  All kernels here are bound by HBM, and on B200 their speed
+// depends on how many bytes each SM keeps in flight: too few starve the memory
+// system, too many make the reads and write-backs of many chunks collide in
+// DRAM (the read+write passes are fastest with ONE CTA per SM and 48-64 KB of
+// reads in flight).  The table holds the measured best per element-type pair:
+//   T     threads per CTA
+//   U     four-element vectors in flight per thread and operand
+//   UK    the same for a step that leaves g alone (only g read, only d written)
+//   C     resident CTAs per SM the grid is sized for (0 = all that fit)
+//   MINB  occupancy asked of the compiler through __launch_bounds__
+// A build that times variants substitutes its own table with
+// -DGAC_GEOMETRY_HEADER='"file.h"'.
+template <typename P>
+struct StatsGeom;   // fused triple reduction
+template <typename P>
+struct ProjGeom;    // projection + state refresh
+template <typename P>
+struct AdamGeom;    // projection fused with AdamW
+#ifdef GAC_GEOMETRY_HEADER
+#include GAC_GEOMETRY_HEADER
+#else
+template <> struct StatsGeom<float>       { static constexpr int T = 256, U = 8, C = 0, MINB = 4; };
+template <> struct StatsGeom<bf16_t>      { static constexpr int T = 256, U = 8, C = 0, MINB = 4; };
+template <> struct StatsGeom<bf16_pair_t> { static constexpr int T = 256, U = 8, C = 0, MINB = 4; };
+template <> struct ProjGeom<float>        { static constexpr int T = 256, U = 8, UK = 16, C = 1, MINB = 1; };
+template <> struct ProjGeom<bf16_t>       { static constexpr int T = 512, U = 4, UK = 8, C = 1, MINB = 1; };
+template <> struct ProjGeom<bf16_pair_t>  { static constexpr int T = 512, U = 8, UK = 8, C = 1, MINB = 1; };
+template <> struct AdamGeom<float>        { static constexpr int T = 1024, U = 1, C = 1; };
+template <> struct AdamGeom<bf16_t>       { static constexpr int T = 1024, U = 1, C = 1; };
+template <> struct AdamGeom<bf16_pair_t>  { static constexpr int T = 1024, U = 1, C = 1; };
+#endif
 
 __device__ __forceinline__ uint32_t pack_bf16x2_rn(float lo, float hi) {
     uint32_t r;
