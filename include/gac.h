@@ -37,7 +37,7 @@ typedef enum {
     GAC_ERR_CUDA = 3,          /* a CUDA runtime call failed; message has the CUDA error     */
     GAC_ERR_STATE = 4,         /* calls out of order (project without stats, step going back)*/
     GAC_ERR_NONFINITE = 5,     /* NaN/Inf met in g or d; the step is reported as a violation  */
-    GAC_ERR_TIMEOUT = 6        /* reserved: no entry point of this library waits on the device */
+    GAC_ERR_TIMEOUT = 6        /* reserved: no kernel of this library waits on a flag or a peer  */
 } gac_status;
 
 typedef enum { GAC_F32 = 0, GAC_BF16 = 1 } gac_dtype;
@@ -230,6 +230,18 @@ const char *gac_last_error(const gac_ctx *ctx);
  * Changing them changes the summation order, hence the last bits of the sums.
  */
 int gac_set_launch(gac_ctx *ctx, int chunk_elems, int ctas_per_sm);
+
+/*
+ * gac_rebind -- point an existing context at moved buffers (a framework that
+ * re-allocates its gradient tensors changes their addresses, not their sizes).
+ * Same number of tensors and the same numel each; the step counter, the
+ * hyper-parameters and the device-resident record are kept, so the state in
+ * the new d buffers is taken as the stored direction of the next step.  Only
+ * between steps (not between gac_stats and gac_project).  Frees and
+ * re-allocates the chunk table, which synchronises the device.
+ * Errors: INVALID_ARG, STATE, CUDA.
+ */
+int gac_rebind(gac_ctx *ctx, const gac_tensor *list, uint32_t n);
 
 /* Facts about the context: total elements, chunks, grid size, kernel launches so far. */
 typedef struct {

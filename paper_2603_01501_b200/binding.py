@@ -68,7 +68,8 @@ class gac_info(ctypes.Structure):
 
 EXPORTS = ["gac_default_hparams", "gac_init", "gac_stats", "gac_stats_partial", "gac_decide",
            "gac_project", "gac_free", "gac_last_error", "gac_set_launch", "gac_get_info",
-           "gac_stats_static", "gac_default_adamw", "gac_attach_adamw", "gac_project_adamw"]
+           "gac_stats_static", "gac_default_adamw", "gac_attach_adamw", "gac_project_adamw",
+           "gac_rebind"]
 
 _lib = None
 
@@ -106,6 +107,8 @@ def load_library() -> ctypes.CDLL:
     L.gac_stats_static.argtypes = [ctypes.POINTER(gac_tensor), u32, i32, i32,
                                    ctypes.POINTER(gac_hparams), u64, u32, i32, vp, vp]
     L.gac_stats_static.restype = i32
+    L.gac_rebind.argtypes = [vp, ctypes.POINTER(gac_tensor), u32]
+    L.gac_rebind.restype = i32
     L.gac_default_adamw.argtypes = [ctypes.POINTER(gac_adamw)]
     L.gac_default_adamw.restype = None
     L.gac_attach_adamw.argtypes = [vp, ctypes.POINTER(gac_opt_tensor), u32, u64]
@@ -331,3 +334,15 @@ def gac_project_adamw(ctx: GacContext, opt: AdamW, stream=None, coef_override: O
                              ctypes.byref(res) if fetch else None)
     ctx._check(rc, allow_nonfinite=True)
     return res
+
+
+def gac_rebind(ctx: GacContext, g_list: Sequence[torch.Tensor], d_list: Sequence[torch.Tensor]) -> None:
+    """Points the context at moved buffers of the same sizes (gac_rebind of the C ABI)."""
+    n = len(g_list)
+    arr = (gac_tensor * max(n, 1))()
+    for i, (g, d) in enumerate(zip(g_list, d_list)):
+        if not (g.is_cuda and d.is_cuda and g.is_contiguous() and d.is_contiguous()):
+            raise ValueError("tensors must be contiguous CUDA tensors")
+        arr[i] = gac_tensor(g.data_ptr(), d.data_ptr(), g.numel())
+    ctx._check(load_library().gac_rebind(ctx.handle, arr, n))
+    ctx._keep = (list(g_list), list(d_list))

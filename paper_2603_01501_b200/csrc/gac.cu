@@ -267,6 +267,38 @@ int check_hparams(const gac_hparams *hp) {
     return GAC_OK;
 }
 
+// Pointer, size and overlap checks of a tensor list (host only).
+int check_list(gac_ctx *ctx, const gac_tensor *list, uint32_t n, size_t gs, size_t ds) {
+    for (uint32_t i = 0; i < n; ++i) {
+        if (!list[i].g || !list[i].d)
+            return fail(ctx, GAC_ERR_INVALID_ARG, "tensor %s%lld has a NULL pointer", "", i);
+        if (list[i].numel == 0)
+            return fail(ctx, GAC_ERR_INVALID_ARG, "tensor %s%lld has no elements", "", i);
+        if (list[i].numel > (1ull << 40))
+            return fail(ctx, GAC_ERR_INVALID_ARG, "tensor %s%lld is larger than 2^40 elements", "", i);
+        const uint64_t gb = reinterpret_cast<uint64_t>(list[i].g), db = reinterpret_cast<uint64_t>(list[i].d);
+        if (gb % gs || db % ds)
+            return fail(ctx, GAC_ERR_INVALID_ARG, "tensor %s%lld is not element-aligned", "", i);
+        // g is updated in place while d is read: the two ranges must not overlap
+        if (gb < db + list[i].numel * ds && db < gb + list[i].numel * gs)
+            return fail(ctx, GAC_ERR_INVALID_ARG, "tensor %s%lld: g and d overlap", "", i);
+    }
+    {   // every g and every d is written in place: all 2n ranges must be pairwise disjoint
+        std::vector<std::pair<uint64_t, uint64_t>> ranges;
+        ranges.reserve(2 * size_t(n));
+        for (uint32_t i = 0; i < n; ++i) {
+            const uint64_t gb = reinterpret_cast<uint64_t>(list[i].g), db = reinterpret_cast<uint64_t>(list[i].d);
+            ranges.emplace_back(gb, gb + list[i].numel * gs);
+            ranges.emplace_back(db, db + list[i].numel * ds);
+        }
+        std::sort(ranges.begin(), ranges.end());
+        for (size_t i = 1; i < ranges.size(); ++i)
+            if (ranges[i].first < ranges[i - 1].second)
+                return fail(ctx, GAC_ERR_INVALID_ARG, "buffers of different tensors overlap%s");
+    }
+    return GAC_OK;
+}
+
 DevHP dev_hp(const gac_ctx *c, uint64_t step, uint32_t staleness, int decide) {
     DevHP h;
     h.c_low = c->hp.c_low;
@@ -337,33 +369,7 @@ int gac_init(gac_ctx **out, const gac_tensor *list, uint32_t n, int g_dtype, int
         return fail(nullptr, GAC_ERR_DTYPE, "supported (g,d) element types: (f32,f32), (bf16,f32), (bf16,bf16)%s");
     if (int rc = check_hparams(hp)) return rc;
     const size_t gs = elem_size(g_dtype), ds = elem_size(d_dtype);
-    for (uint32_t i = 0; i < n; ++i) {
-        if (!list[i].g || !list[i].d)
-            return fail(nullptr, GAC_ERR_INVALID_ARG, "tensor %s%lld has a NULL pointer", "", i);
-        if (list[i].numel == 0)
-            return fail(nullptr, GAC_ERR_INVALID_ARG, "tensor %s%lld has no elements", "", i);
-        if (list[i].numel > (1ull << 40))
-            return fail(nullptr, GAC_ERR_INVALID_ARG, "tensor %s%lld is larger than 2^40 elements", "", i);
-        const uint64_t gb = reinterpret_cast<uint64_t>(list[i].g), db = reinterpret_cast<uint64_t>(list[i].d);
-        if (gb % gs || db % ds)
-            return fail(nullptr, GAC_ERR_INVALID_ARG, "tensor %s%lld is not element-aligned", "", i);
-        // g is updated in place while d is read: the two ranges must not overlap
-        if (gb < db + list[i].numel * ds && db < gb + list[i].numel * gs)
-            return fail(nullptr, GAC_ERR_INVALID_ARG, "tensor %s%lld: g and d overlap", "", i);
-    }
-    {   // every g and every d is written in place: all 2n ranges must be pairwise disjoint
-        std::vector<std::pair<uint64_t, uint64_t>> ranges;
-        ranges.reserve(2 * size_t(n));
-        for (uint32_t i = 0; i < n; ++i) {
-            const uint64_t gb = reinterpret_cast<uint64_t>(list[i].g), db = reinterpret_cast<uint64_t>(list[i].d);
-            ranges.emplace_back(gb, gb + list[i].numel * gs);
-            ranges.emplace_back(db, db + list[i].numel * ds);
-        }
-        std::sort(ranges.begin(), ranges.end());
-        for (size_t i = 1; i < ranges.size(); ++i)
-            if (ranges[i].first < ranges[i - 1].second)
-                return fail(nullptr, GAC_ERR_INVALID_ARG, "buffers of different tensors overlap%s");
-    }
+    if (int rc = check_list(nullptr, list, n, gs, ds)) return rc;
     int n_dev = 0;
     if (cudaGetDeviceCount(&n_dev) != cudaSuccess || n_dev == 0)
         return fail(nullptr, GAC_ERR_CUDA, "no CUDA device is available%s");
@@ -417,6 +423,21 @@ int gac_set_launch(gac_ctx *ctx, int chunk_elems, int ctas_per_sm) {
     }
     if (ctas_per_sm > 0) ctx->ctas_per_sm = std::min(ctas_per_sm, kMaxCtasPerSm);
     DeviceGuard guard(ctx->device);
+    return build_table(ctx);
+}
+
+int gac_rebind(gac_ctx *ctx, const gac_tensor *list, uint32_t n) {
+    if (!ctx) return fail(nullptr, GAC_ERR_INVALID_ARG, "ctx is NULL%s");
+    if (!list || n != ctx->list.size())
+        return fail(ctx, GAC_ERR_INVALID_ARG, "gac_rebind needs one entry per tensor of the context%s");
+    for (uint32_t i = 0; i < n; ++i)
+        if (list[i].numel != ctx->list[i].numel)
+            return fail(ctx, GAC_ERR_INVALID_ARG, "tensor %s%lld changed its element count; create a new context", "", i);
+    if (ctx->stats_pending || ctx->decision_ready)
+        return fail(ctx, GAC_ERR_STATE, "gac_rebind between gac_stats and gac_project would split a step%s");
+    if (int rc = check_list(ctx, list, n, elem_size(ctx->g_dt), elem_size(ctx->d_dt))) return rc;
+    DeviceGuard guard(ctx->device);
+    ctx->list.assign(list, list + n);
     return build_table(ctx);
 }
 

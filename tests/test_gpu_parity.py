@@ -445,3 +445,30 @@ def test_state_recurrence_is_bitwise_and_survives_a_new_context():
         r3 = gb.gac_stats(ctx, 7)
         assert r3.dd == r2.gg and r3.step == 7
         gb.gac_free(ctx)
+
+
+def test_rebind_to_moved_buffers_keeps_the_step_sequence():
+    shapes = synth.decoder_tensor_list(synth.DIMS["mini"])
+    g, d = synth.gradient_list(shapes, 0.4, config_id=2, device="cuda")
+    hp = gb.HParams(**FORCE)
+    ctx = gb.gac_init(g, d, hp)
+    gb.gac_stats(ctx, 2)
+    with pytest.raises(gb.GacError) as e:
+        gb.gac_rebind(ctx, g, d)                       # a step is open
+    assert e.value.status == gb.GAC_ERR_STATE
+    gb.gac_project(ctx)
+    torch.cuda.synchronize()
+    g2 = [torch.randn_like(t) * 0.01 for t in g]        # the framework re-allocated its gradients
+    d2 = [t.clone() for t in d]                         # ... and the snapshot moved with them
+    gb.gac_rebind(ctx, g2, d2)
+    g_ref, d_ref = [t.cpu() for t in g2], [t.cpu() for t in d2]
+    dec = orc.step(g_ref, d_ref, to_orc_hp(hp))
+    res = gb.gac_stats(ctx, 3)
+    gb.gac_project(ctx, coef_override=dec.coef if dec.regime == orc.PROJECT else None)
+    torch.cuda.synchronize()
+    check_sums(res, dec)
+    check_decision(res, dec)
+    check_outputs(g2, d2, g_ref, d_ref)
+    with pytest.raises(gb.GacError):
+        gb.gac_rebind(ctx, g2[:-1], d2[:-1])
+    gb.gac_free(ctx)
