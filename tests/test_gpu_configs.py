@@ -200,3 +200,39 @@ def test_staleness_run_full_size_sample():
         log = staleness_run(shapes, rho, k, run_id=900 + k, steps=steps, hp=band, full_outputs=False)
         assert log[0][1] == gb.GAC_REGIME_SAFE
         assert any(r == gb.GAC_REGIME_PROJECT for _, r, _ in log[1:]) or rho == 0.0
+
+
+def test_single_tensor_beyond_32bit_indexing():
+    """One tensor of 2^32 + 4099 elements (bfloat16 pair, 8.6 GB per buffer): element offsets do not
+    fit 32 bits; sums over all of it, outputs on slices around the 2^32 boundary and at both ends."""
+    n = (1 << 32) + 4099
+    free, _ = torch.cuda.mem_get_info()
+    if free < (40 << 30):
+        pytest.skip("needs 40 GiB of device memory")
+    gen = torch.Generator(device="cuda").manual_seed(99)
+    d = torch.empty(n, dtype=torch.bfloat16, device="cuda")
+    g = torch.empty(n, dtype=torch.bfloat16, device="cuda")
+    step = 1 << 28
+    for lo in range(0, n, step):            # generated piecewise to bound temporaries
+        hi = min(n, lo + step)
+        z = torch.randn(hi - lo, generator=gen, device="cuda")
+        w = torch.randn(hi - lo, generator=gen, device="cuda")
+        d[lo:hi] = (0.01 * z).to(torch.bfloat16)
+        g[lo:hi] = (0.005 * z + 0.00866 * w).to(torch.bfloat16)
+    g0, d0 = g.clone(), d.clone()
+    hp = gb.HParams(**FORCE)
+    dec = orc.decide(oracle_sums_streamed([g], [d]), to_orc_hp(hp))
+    ctx = gb.gac_init([g], [d], hp)
+    res = gb.gac_stats(ctx, 2)
+    gb.gac_project(ctx, coef_override=dec.coef)
+    torch.cuda.synchronize()
+    gb.gac_free(ctx)
+    check_sums(res, dec)
+    check_decision(res, dec)
+    assert dec.regime == orc.PROJECT and abs(res.cos - 0.5) < 0.01
+    assert torch.equal(d.view(torch.int16), g0.view(torch.int16))       # state = raw gradient, every element
+    for lo, hi in [(0, SLICE), ((1 << 32) - SLICE // 2 - 1, (1 << 32) + 4099), ((1 << 31) + 1, (1 << 31) + SLICE)]:
+        g_ref, d_ref = g0[lo:hi].cpu().contiguous(), d0[lo:hi].cpu().contiguous()
+        orc.project([g_ref], [d_ref], to_orc_hp(hp), dec, threads=THREADS)
+        assert max_ulp(g[lo:hi].cpu(), g_ref) <= 1
+        assert torch.equal(d[lo:hi].cpu().view(torch.int16), d_ref.view(torch.int16))
