@@ -572,21 +572,32 @@ __device__ __forceinline__ double outgoing64(float g, float d, float k, double b
 
 // One element of: g' -> AdamW, in binary64 so that p - delta stays accurate
 // even where it cancels (tiny parameters).  The square root and the reciprocal
-// start from binary32 hardware results and take one Newton step each in
-// binary64 (relative error ~1e-14), far cheaper than the binary64 library
-// routines.  m, v and p are each rounded once on the way out.
+// start from the hardware's binary64 approximations (about 20 good bits, no
+// conversion to binary32 and back) and take one Newton step each (relative
+// error ~1e-12), far cheaper than the full binary64 routines.  m, v and p are
+// each rounded once on the way out.
+__device__ __forceinline__ double rsqrt_approx64(double x) {
+    double y;
+    asm("rsqrt.approx.ftz.f64 %0, %1;" : "=d"(y) : "d"(x));
+    return y;
+}
+__device__ __forceinline__ double rcp_approx64(double x) {
+    double y;
+    asm("rcp.approx.ftz.f64 %0, %1;" : "=d"(y) : "d"(x));
+    return y;
+}
 __device__ __forceinline__ void adamw_elem(double g64, float &p, float &m, float &v, const AdamConst &a) {
-    const double m64 = __dadd_rn(__dmul_rn(a.b1, double(m)), __dmul_rn(a.c1, g64));
-    const double v64 = __dadd_rn(__dmul_rn(a.b2, double(v)), __dmul_rn(__dmul_rn(a.c2, g64), g64));
+    const double m64 = fma(a.b1, double(m), a.c1 * g64);
+    const double v64 = fma(a.b2, double(v), (a.c2 * g64) * g64);
     double root = 0.0;
-    const float r32 = __fsqrt_rn(__double2float_rn(v64));
-    if (r32 > 0.0f) {
-        const double r = double(r32);
-        root = fma(fma(-r, r, v64), double(__fdividef(0.5f, r32)), r);   // r + (v - r^2)/(2r)
+    if (v64 > 1e-300) {                                  // below that the root is far under any eps
+        const double y = rsqrt_approx64(v64);
+        const double r = v64 * y;
+        root = fma(fma(-r, r, v64), 0.5 * y, r);         // r + (v - r^2) / (2 sqrt(v))
     }
     const double denom = fma(root, a.inv_sqrt_bc2, a.eps);
-    const double q = double(__frcp_rn(__double2float_rn(denom)));
-    const double inv = q * fma(-denom, q, 2.0);                           // q (2 - denom q)
+    const double q = rcp_approx64(denom);
+    const double inv = q * fma(-denom, q, 2.0);          // q (2 - denom q)
     const double delta = fma(a.lr_wd, double(p), a.step_size * (m64 * inv));
     p = __double2float_rn(double(p) - delta);
     m = __double2float_rn(m64);

@@ -10,7 +10,7 @@ from oracle import gac_oracle as orc
 from paper_2603_01501_b200 import binding as gb
 from paper_2603_01501_b200 import synth
 
-from gpu_util import check_decision, check_sums, max_ulp, to_orc_hp
+from gpu_util import check_decision, check_sums, max_ulp, ordered_int, to_orc_hp
 
 pytestmark = pytest.mark.gpu
 
@@ -42,6 +42,8 @@ def run_sequence(g_dtype, hp, opt_kw, shapes_name="mini", rhos=(None, 0.0, 0.3, 
             dst.copy_(src)
         first = t == 1
         dec = orc.decide(orc.stats(g, d_cpu, first_step=first), ohp, first)
+        m_before = [x.clone() for x in m_cpu]
+        d_before = [x.clone().float() for x in d_cpu]
         did = orc.project_adamw(g, d_cpu, p_cpu, m_cpu, v_cpu, ohp, dec, oopt, applied + 1, first)
         applied += int(did)
         res = gb.gac_stats(ctx, t)
@@ -53,13 +55,27 @@ def run_sequence(g_dtype, hp, opt_kw, shapes_name="mini", rhos=(None, 0.0, 0.3, 
         if hp.clip_max_norm > 0 and dec.regime != orc.VIOLATION:
             assert abs(after.clip_scale - dec.clip_scale) <= 1e-9 * dec.clip_scale
         for i in range(n_t):
-            assert torch.equal(g_gpu[i].cpu().view(torch.int16 if g_dtype == torch.bfloat16 else torch.int32),
-                               g[i].view(torch.int16 if g_dtype == torch.bfloat16 else torch.int32)), "g was written"
+            bits = torch.int16 if g_dtype == torch.bfloat16 else torch.int32
+            assert torch.equal(g_gpu[i].cpu().view(bits), g[i].view(bits)), "g was written"
             assert torch.equal(d_gpu[i].cpu(), d_cpu[i]), "stored direction is not the raw gradient"
-            for name, a, b in (("p", p_gpu[i], p_cpu[i]), ("m", m_gpu[i], m_cpu[i]), ("v", v_gpu[i], v_cpu[i])):
-                u = max_ulp(a.cpu(), b)
-                assert u <= 4, f"step {t} tensor {i} {name}: {u} ulp"
-                worst = max(worst, u)
+            # v is a sum of non-negative terms: plain ulp distance.  m = b1 m + (1-b1) g' and
+            # p = p - delta can cancel (with bfloat16 gradients even exactly), so where they do the
+            # bound is the rounding noise of the binary64 terms instead of ulps of the tiny result.
+            gmag = g[i].float().abs() + abs(dec.coef) * d_before[i].abs().nan_to_num(0.0)
+            checks = (("v", v_gpu[i], v_cpu[i], None),
+                      ("m", m_gpu[i], m_cpu[i], 1e-13 * (m_before[i].abs() + gmag)),
+                      ("p", p_gpu[i], p_cpu[i], torch.full_like(p_cpu[i], 1e-10 * oopt.lr)))
+            for name, a, b, slack in checks:
+                a_cpu = a.cpu()
+                ulps = (ordered_int(a_cpu) - ordered_int(b)).abs()
+                ok = ulps <= 4
+                if slack is not None:
+                    ok |= (a_cpu.double() - b.double()).abs() <= slack.double()
+                assert bool(ok.all()), f"step {t} tensor {i} {name}: {int(ulps[~ok].max())} ulp"
+                worst = max(worst, int(ulps[ok & (ulps <= 4)].max()) if bool((ulps <= 4).any()) else 0)
+                # each step is compared from identical state: a last-bit difference (a rounding tie
+                # taken the other way) would otherwise be carried into later steps
+                a.copy_(b)
         regimes.append(dec.regime)
     gb.gac_free(ctx)
     return regimes, applied, worst
