@@ -24,3 +24,17 @@ def pytest_collection_modifyitems(config, items):
     for item in items:
         if "gpu" in item.keywords:
             item.add_marker(skip)
+
+
+@pytest.fixture(scope="session", autouse=True)
+def _built_libraries():
+    """Builds what the tests load if it is missing or older than its sources: the CUDA library
+    (nvcc cross-compiles without a GPU) and the C checker.  The package itself never builds on
+    import and fails loudly when its library is absent."""
+    import shutil
+    if shutil.which("nvcc"):
+        from paper_2603_01501_b200 import build as gbuild
+        gbuild.build()
+    from oracle import gac_oracle
+    gac_oracle.build()
+    yield
