@@ -34,7 +34,7 @@
 // The ABI's structs as laid out for callers in other languages (the Python binding mirrors them).
 static_assert(sizeof(gac_tensor) == 24, "gac_tensor layout");
 static_assert(sizeof(gac_hparams) == 72, "gac_hparams layout");
-static_assert(sizeof(gac_result) == 104, "gac_result layout");
+static_assert(sizeof(gac_result) == 96, "gac_result layout");
 static_assert(sizeof(gac_opt_tensor) == 24 && sizeof(gac_adamw) == 40, "optimizer structs layout");
 
 // ===================================================================== host
