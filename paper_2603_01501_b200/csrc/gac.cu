@@ -618,6 +618,7 @@ struct StaticSetup {
 };
 StaticSetup g_static_setup[kMaxDevices];
 std::mutex g_static_mutex;
+Chunk g_static_host_table[kStaticMaxChunks];   // host image of the chunk table, filled under the mutex
 
 // Runs once per device, with that device current.  The array's name is only a
 // host-side handle here; the address a kernel can use comes from the runtime.
@@ -681,32 +682,33 @@ extern "C" int gac_stats_static(const gac_tensor *list, uint32_t n, int g_dtype,
     StaticSetup *st = nullptr;
     if (int rc = static_setup(cuda_device, &st)) return rc;
 
-    // host-side image of the table (host memory only), then one copy into the scratch
-    static thread_local std::vector<Chunk> table;
-    table.clear();
-    table.reserve(n_chunks);
-    for (uint32_t i = 0; i < n; ++i) {
-        const uint64_t gb = reinterpret_cast<uint64_t>(list[i].g), db = reinterpret_cast<uint64_t>(list[i].d);
-        const bool aligned = (gb % 16 == 0) && (db % 16 == 0);
-        for (uint64_t off = 0; off < list[i].numel; off += ce) {
-            Chunk ch;
-            ch.g = gb + off * gs;
-            ch.d = db + off * ds;
-            ch.n = uint32_t(std::min<uint64_t>(ce, list[i].numel - off));
-            ch.flags = aligned ? kChunkAligned : 0u;
-            ch.pad = 0;
-            table.push_back(ch);
-        }
-    }
+    // Host-side image of the table in a fixed buffer of the library (no heap use either), then one
+    // copy into the device scratch.  The lock covers filling and staging: the copy call returns once
+    // the pageable source has been staged, after which the buffer may be refilled by another caller.
     cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
     Chunk *d_chunks = reinterpret_cast<Chunk *>(st->base + kStaticChunksOff);
     double *d_partials = reinterpret_cast<double *>(st->base + kStaticPartialsOff);
     unsigned *d_ticket = reinterpret_cast<unsigned *>(st->base + kStaticTicketOff);
-    // the scratch keeps whatever the previous call left: the ticket must start at zero
-    GAC_CUDA(nullptr, cudaMemsetAsync(d_ticket, 0, sizeof(unsigned), s));
-    // source is pageable host memory: the call returns once it has been staged, so `table` may be reused
-    GAC_CUDA(nullptr, cudaMemcpyAsync(d_chunks, table.data(), table.size() * sizeof(Chunk),
-                                      cudaMemcpyHostToDevice, s));
+    {
+        std::lock_guard<std::mutex> lock(g_static_mutex);
+        uint64_t filled = 0;
+        for (uint32_t i = 0; i < n; ++i) {
+            const uint64_t gb = reinterpret_cast<uint64_t>(list[i].g), db = reinterpret_cast<uint64_t>(list[i].d);
+            const bool aligned = (gb % 16 == 0) && (db % 16 == 0);
+            for (uint64_t off = 0; off < list[i].numel; off += ce) {
+                Chunk &ch = g_static_host_table[filled++];
+                ch.g = gb + off * gs;
+                ch.d = db + off * ds;
+                ch.n = uint32_t(std::min<uint64_t>(ce, list[i].numel - off));
+                ch.flags = aligned ? kChunkAligned : 0u;
+                ch.pad = 0;
+            }
+        }
+        // the scratch keeps whatever the previous call left: the ticket must start at zero
+        GAC_CUDA(nullptr, cudaMemsetAsync(d_ticket, 0, sizeof(unsigned), s));
+        GAC_CUDA(nullptr, cudaMemcpyAsync(d_chunks, g_static_host_table, filled * sizeof(Chunk),
+                                          cudaMemcpyHostToDevice, s));
+    }
     gac_ctx shell;            // only carries the hyper-parameters into dev_hp()
     shell.hp = *hp;
     const DevHP h = dev_hp(&shell, step, staleness, 1);
