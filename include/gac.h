@@ -268,7 +268,9 @@ int gac_get_info(const gac_ctx *ctx, gac_info *out);
  * where the implicit device-wide synchronisation of cudaMalloc/cudaFree is
  * unacceptable, or in a process that was told to keep a fixed memory footprint.
  * gac_init allocates a chunk table, partial sums and a pinned mirror; this
- * entry point needs no context and calls no allocating CUDA routine at all.
+ * entry point needs no context, calls no allocating CUDA routine and does not
+ * use the host heap either (the host image of the table sits in a fixed 2 MiB
+ * buffer of the library, filled under a lock).
  *
  * How: the chunk table, the per-CTA partial sums and the arrival ticket live
  * in an array that is part of the library image: GAC_STATIC_SCRATCH_BYTES
