@@ -46,7 +46,16 @@ typedef enum { GAC_F32 = 0, GAC_BF16 = 1 } gac_dtype;
 typedef enum { GAC_REGIME_SAFE = 0, GAC_REGIME_PROJECT = 1, GAC_REGIME_VIOLATION = 2 } gac_regime;
 
 typedef enum { GAC_MODE_ADAPTIVE = 0, GAC_MODE_FIXED = 1 } gac_mode;
-typedef enum { GAC_STATE_RAW = 0, GAC_STATE_PROJECTED = 1, GAC_STATE_HOLD = 2 } gac_state_mode;
+typedef enum {
+    GAC_STATE_RAW = 0,        /* d' = g, copied into the d buffers (the paper's rule)            */
+    GAC_STATE_PROJECTED = 1,  /* d' = g' (variant)                                               */
+    GAC_STATE_HOLD = 2,       /* d' = d  (variant)                                               */
+    GAC_STATE_EXCHANGE = 3    /* d' = g as in RAW, but WITHOUT the copy: the two buffer sets swap
+                                 roles after every step (see "Exchange mode" below)              */
+} gac_state_mode;
+
+/* Which of the two buffer sets of a context's list: the `g` pointers or the `d` pointers. */
+typedef enum { GAC_SET_G = 0, GAC_SET_D = 1 } gac_buffer_set;
 
 /* One parameter tensor: its gradient and its slot of the stored direction.
  * Both are device pointers to `numel` contiguous elements, caller-owned.
@@ -68,7 +77,7 @@ typedef struct {
     int32_t mode;              /* gac_mode: ADAPTIVE = Eq. 5 with the three regimes;
                                   FIXED = Eq. 3 with (alpha_fixed, beta) on every step         */
     int32_t state_mode;        /* gac_state_mode: RAW d' = g (the paper's rule);
-                                  PROJECTED d' = g'; HOLD d' = d                                */
+                                  PROJECTED d' = g'; HOLD d' = d; EXCHANGE d' = g by role swap  */
     double alpha_fixed;        /* gain of the parallel component in FIXED mode; 0 = remove it   */
     int32_t zero_on_violation; /* 0: leave g alone, the caller skips its optimizer step
                                   (Algorithm 1: theta_t = theta_{t-1}); 1: write g' = 0          */
@@ -101,6 +110,15 @@ typedef struct {
     double clip_scale;         /* factor applied by clipping (1 when off, not needed, or skipped) */
     uint64_t applied_steps;    /* optimizer updates applied so far by gac_project_adamw (skipped steps
                                   do not count); kept on the device across steps                  */
+    uint32_t g_set;            /* gac_buffer_set that held this step's gradient (always GAC_SET_G
+                                  outside exchange mode)                                          */
+    uint32_t out_set;          /* gac_buffer_set that holds what the step sends on after
+                                  gac_project: the same as g_set when g is updated in place or
+                                  left alone; the other set when exchange mode wrote g' there     */
+    uint32_t ref_lost;         /* exchange mode only: a non-finite step was closed, the stored
+                                  direction is gone and the next step restarts from the zero
+                                  reference (Algorithm 1's g_0 = 0)                               */
+    uint32_t reserved;
 } gac_result;
 
 /* Fills *hp with the paper's defaults. */
@@ -181,6 +199,32 @@ int gac_decide(gac_ctx *ctx, void *cuda_stream, const double *sums_in, gac_resul
 int gac_project(gac_ctx *ctx, void *cuda_stream, const float *coef_override, gac_result *host_out);
 
 /*
+ * Exchange mode (state_mode GAC_STATE_EXCHANGE; g and d of the SAME element type).
+ * App. A.2 keeps one snapshot of the previous gradient; refreshing it by a copy
+ * costs a write of the whole vector on every step.  Here nothing is copied: the
+ * buffers that held g simply BECOME the stored direction (they hold the raw
+ * gradient already), and the buffers that held d become free.
+ *   projection step   g' is written into the buffers that held d (read g, read d,
+ *                     write once: 3 instead of 4 element transfers per parameter);
+ *                     g itself is not modified
+ *   safe / violation  nothing is read or written in the second pass; what a safe
+ *                     step sends on is g, where it lies (read it, do not modify
+ *                     it: it is the stored direction now).  zero_on_violation and
+ *                     an active clip factor write their result (0, or s g) into
+ *                     the buffers that held d.
+ * After every gac_project / gac_project_adamw the roles swap: the NEXT gradient
+ * must be written into the set that held d during this step.  The swap is
+ * unconditional, so the caller can follow it without reading anything back:
+ * step by step the gradient alternates between the two sets, starting with the
+ * `g` pointers given to gac_init (gac_rebind starts over with the new `g`).
+ * gac_next_gradient_set reports it.  The record says where the outgoing gradient
+ * is (`out_set`).  A non-finite step writes nothing; since the roles swap all the
+ * same, the stored direction is lost with it and the following step is taken
+ * against the zero reference (`ref_lost`), as the first step is.
+ */
+int gac_next_gradient_set(const gac_ctx *ctx, int *set_out /* host pointer: gac_buffer_set */);
+
+/*
  * The step after the path: the update handed straight to the optimizer.
  * Algorithm 1 ends each safe or projection step with theta_t = theta_{t-1} +
  * eta g' and the paper trains with AdamW (Table 2: lr 1e-6, betas (0.9, 0.999),
@@ -199,7 +243,8 @@ int gac_project(gac_ctx *ctx, void *cuda_stream, const float *coef_override, gac
  *                    owned) and sets the number of updates applied so far
  *                    (0 for a fresh optimizer).  Allocates a second table.
  * gac_project_adamw  replaces gac_project for this step (same call order rules).
- *                    Needs state_mode RAW.  opt is a host pointer, copied.
+ *                    Needs state_mode RAW or EXCHANGE (then d' is not written either:
+ *                    the roles swap).  opt is a host pointer, copied.
  * Errors: INVALID_ARG, STATE (not attached, no decision pending), CUDA.
  */
 typedef struct {

@@ -21,7 +21,8 @@ GAC_OK, GAC_ERR_INVALID_ARG, GAC_ERR_DTYPE, GAC_ERR_CUDA, GAC_ERR_STATE, GAC_ERR
 GAC_F32, GAC_BF16 = 0, 1
 GAC_REGIME_SAFE, GAC_REGIME_PROJECT, GAC_REGIME_VIOLATION = 0, 1, 2
 GAC_MODE_ADAPTIVE, GAC_MODE_FIXED = 0, 1
-GAC_STATE_RAW, GAC_STATE_PROJECTED, GAC_STATE_HOLD = 0, 1, 2
+GAC_STATE_RAW, GAC_STATE_PROJECTED, GAC_STATE_HOLD, GAC_STATE_EXCHANGE = 0, 1, 2, 3
+GAC_SET_G, GAC_SET_D = 0, 1
 REGIME_NAMES = {0: "safe", 1: "project", 2: "violation"}
 
 
@@ -43,7 +44,9 @@ class gac_result(ctypes.Structure):
                 ("coef", ctypes.c_float), ("regime", ctypes.c_int32), ("nonfinite", ctypes.c_int32),
                 ("staleness", ctypes.c_uint32), ("step", ctypes.c_uint64),
                 ("out_norm", ctypes.c_double), ("clip_scale", ctypes.c_double),
-                ("applied_steps", ctypes.c_uint64)]
+                ("applied_steps", ctypes.c_uint64), ("g_set", ctypes.c_uint32),
+                ("out_set", ctypes.c_uint32), ("ref_lost", ctypes.c_uint32),
+                ("reserved", ctypes.c_uint32)]
 
     def as_dict(self):
         return {k: getattr(self, k) for k, _ in self._fields_}
@@ -69,7 +72,7 @@ class gac_info(ctypes.Structure):
 EXPORTS = ["gac_default_hparams", "gac_init", "gac_stats", "gac_stats_partial", "gac_decide",
            "gac_project", "gac_free", "gac_last_error", "gac_set_launch", "gac_get_info",
            "gac_stats_static", "gac_default_adamw", "gac_attach_adamw", "gac_project_adamw",
-           "gac_rebind"]
+           "gac_rebind", "gac_next_gradient_set"]
 
 _lib = None
 
@@ -109,6 +112,8 @@ def load_library() -> ctypes.CDLL:
     L.gac_stats_static.restype = i32
     L.gac_rebind.argtypes = [vp, ctypes.POINTER(gac_tensor), u32]
     L.gac_rebind.restype = i32
+    L.gac_next_gradient_set.argtypes = [vp, ctypes.POINTER(ctypes.c_int)]
+    L.gac_next_gradient_set.restype = i32
     L.gac_default_adamw.argtypes = [ctypes.POINTER(gac_adamw)]
     L.gac_default_adamw.restype = None
     L.gac_attach_adamw.argtypes = [vp, ctypes.POINTER(gac_opt_tensor), u32, u64]
@@ -245,6 +250,13 @@ def gac_project(ctx: GacContext, stream=None, coef_override: Optional[float] = N
                        ctypes.byref(res) if fetch else None)
     ctx._check(rc, allow_nonfinite=True)
     return res
+
+
+def gac_next_gradient_set(ctx: GacContext) -> int:
+    """Exchange mode: GAC_SET_G or GAC_SET_D, the buffer set the next gradient belongs in."""
+    out = ctypes.c_int(0)
+    ctx._check(load_library().gac_next_gradient_set(ctx.handle, ctypes.byref(out)))
+    return out.value
 
 
 def gac_free(ctx: GacContext) -> None:

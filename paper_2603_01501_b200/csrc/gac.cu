@@ -34,7 +34,7 @@
 // The ABI's structs as laid out for callers in other languages (the Python binding mirrors them).
 static_assert(sizeof(gac_tensor) == 24, "gac_tensor layout");
 static_assert(sizeof(gac_hparams) == 72, "gac_hparams layout");
-static_assert(sizeof(gac_result) == 96, "gac_result layout");
+static_assert(sizeof(gac_result) == 112, "gac_result layout");
 static_assert(sizeof(gac_opt_tensor) == 24 && sizeof(gac_adamw) == 40, "optimizer structs layout");
 
 // ===================================================================== host
@@ -71,6 +71,7 @@ struct gac_ctx {
     bool stats_pending = false;    // a partial reduction waits for gac_decide
     bool decision_ready = false;   // a decision waits for gac_project
     bool started = false;
+    int swapped = 0;               // exchange mode: 1 while the list's `d` pointers hold the gradient
     uint64_t launches = 0;
     char err[512] = {0};
 };
@@ -151,7 +152,7 @@ auto with_pair(int pair, F f) {
 
 using StatsKernel = void (*)(const Chunk *, uint32_t, double *, unsigned *, gac_result *, double *, DevHP);
 using AdamKernel = void (*)(const Chunk *, const OptChunk *, uint32_t, gac_result *, unsigned *, float, int,
-                            double, double, double, AdamDev);
+                            double, double, double, AdamDev, int);
 
 StatsKernel stats_kernel_of(int pair) {
     return with_pair(pair, [](auto tag) -> StatsKernel { return gac_stats_kernel<decltype(tag)>; });
@@ -236,6 +237,7 @@ int build_table(gac_ctx *c) {
     ProjectKernel pk = with_pair(c->pair, [=](auto tag) -> ProjectKernel {
         return pick_project<decltype(tag)>(state_mode, beta1, zero);
     });
+    if (!pk) return fail(c, GAC_ERR_DTYPE, "no projection kernel for this state mode and element-type pair%s");
     c->project_fn = reinterpret_cast<const void *>(pk);
     int occ_p = resident_ctas(pk, c->threads_project);
     const int cap_s = stats_cap_of(c->pair);
@@ -263,7 +265,7 @@ int check_hparams(const gac_hparams *hp) {
     } else {
         return fail(nullptr, GAC_ERR_INVALID_ARG, "unknown mode%s");
     }
-    if (hp->state_mode < GAC_STATE_RAW || hp->state_mode > GAC_STATE_HOLD)
+    if (hp->state_mode < GAC_STATE_RAW || hp->state_mode > GAC_STATE_EXCHANGE)
         return fail(nullptr, GAC_ERR_INVALID_ARG, "unknown state_mode%s");
     if (hp->zero_on_violation != 0 && hp->zero_on_violation != 1)
         return fail(nullptr, GAC_ERR_INVALID_ARG, "zero_on_violation must be 0 or 1%s");
@@ -321,6 +323,7 @@ DevHP dev_hp(const gac_ctx *c, uint64_t step, uint32_t staleness, int decide) {
     h.decide = decide;
     h.clip_max = c->hp.clip_max_norm;
     h.clip_eps = c->hp.clip_eps;
+    h.swapped = c->swapped;
     return h;
 }
 
@@ -374,6 +377,8 @@ int gac_init(gac_ctx **out, const gac_tensor *list, uint32_t n, int g_dtype, int
     if (pair_id(g_dtype, d_dtype) < 0)
         return fail(nullptr, GAC_ERR_DTYPE, "supported (g,d) element types: (f32,f32), (bf16,f32), (bf16,bf16)%s");
     if (int rc = check_hparams(hp)) return rc;
+    if (hp->state_mode == GAC_STATE_EXCHANGE && g_dtype != d_dtype)
+        return fail(nullptr, GAC_ERR_DTYPE, "exchange mode swaps the roles of the g and d buffers: both need one element type%s");
     const size_t gs = elem_size(g_dtype), ds = elem_size(d_dtype);
     if (int rc = check_list(nullptr, list, n, gs, ds)) return rc;
     int n_dev = 0;
@@ -444,6 +449,7 @@ int gac_rebind(gac_ctx *ctx, const gac_tensor *list, uint32_t n) {
     if (int rc = check_list(ctx, list, n, elem_size(ctx->g_dt), elem_size(ctx->d_dt))) return rc;
     DeviceGuard guard(ctx->device);
     ctx->list.assign(list, list + n);
+    ctx->swapped = 0;   // exchange mode starts over: the new `g` pointers hold the next gradient
     return build_table(ctx);
 }
 
@@ -496,11 +502,12 @@ int gac_project(gac_ctx *ctx, void *cuda_stream, const float *coef_override, gac
     const int use = coef_override ? 1 : 0;
     const uint32_t nc = uint32_t(ctx->n_chunks);
     reinterpret_cast<ProjectKernel>(const_cast<void *>(ctx->project_fn))<<<ctx->grid_project, ctx->threads_project, 0, s>>>(
-        ctx->d_chunks, nc, ctx->d_rec, k, use, ctx->hp.beta, ctx->hp.clip_max_norm, ctx->hp.clip_eps);
+        ctx->d_chunks, nc, ctx->d_rec, k, use, ctx->hp.beta, ctx->hp.clip_max_norm, ctx->hp.clip_eps, ctx->swapped);
     GAC_CUDA(ctx, cudaGetLastError());
     ++ctx->launches;
     ctx->decision_ready = false;
     ctx->last_projected_step = ctx->pending_step;
+    if (ctx->hp.state_mode == GAC_STATE_EXCHANGE) ctx->swapped ^= 1;   // the buffers that held g are the stored direction now
     return host_out ? read_back(ctx, s, host_out) : GAC_OK;
 }
 
@@ -517,8 +524,8 @@ int gac_attach_adamw(gac_ctx *ctx, const gac_opt_tensor *list, uint32_t n, uint6
     if (!ctx) return fail(nullptr, GAC_ERR_INVALID_ARG, "ctx is NULL%s");
     if (!list || n != ctx->list.size())
         return fail(ctx, GAC_ERR_INVALID_ARG, "optimizer state list must have one entry per tensor of the context%s");
-    if (ctx->hp.state_mode != GAC_STATE_RAW)
-        return fail(ctx, GAC_ERR_INVALID_ARG, "the fused optimizer step needs state_mode RAW%s");
+    if (ctx->hp.state_mode != GAC_STATE_RAW && ctx->hp.state_mode != GAC_STATE_EXCHANGE)
+        return fail(ctx, GAC_ERR_INVALID_ARG, "the fused optimizer step needs state_mode RAW or EXCHANGE%s");
     for (uint32_t i = 0; i < n; ++i) {
         const void *ptrs[3] = {list[i].p, list[i].m, list[i].v};
         for (const void *q : ptrs) {
@@ -552,13 +559,18 @@ int gac_project_adamw(gac_ctx *ctx, void *cuda_stream, const gac_adamw *opt, con
     const int use = coef_override ? 1 : 0;
     const uint32_t nc = uint32_t(ctx->n_chunks);
     const AdamDev o{opt->lr, opt->beta1, opt->beta2, opt->eps, opt->weight_decay};
-    const AdamKernel ak = with_pair(ctx->pair, [](auto tag) -> AdamKernel { return gac_adamw_kernel<decltype(tag)>; });
+    const bool exch = (ctx->hp.state_mode == GAC_STATE_EXCHANGE);
+    const AdamKernel ak = with_pair(ctx->pair, [exch](auto tag) -> AdamKernel {
+        return exch ? gac_adamw_kernel<decltype(tag), true> : gac_adamw_kernel<decltype(tag), false>;
+    });
     ak<<<ctx->grid_adamw, ctx->threads_adamw, 0, s>>>(ctx->d_chunks, ctx->d_opt_chunks, nc, ctx->d_rec, ctx->d_ticket,
-                                                      k, use, ctx->hp.beta, ctx->hp.clip_max_norm, ctx->hp.clip_eps, o);
+                                                      k, use, ctx->hp.beta, ctx->hp.clip_max_norm, ctx->hp.clip_eps, o,
+                                                      ctx->swapped);
     GAC_CUDA(ctx, cudaGetLastError());
     ++ctx->launches;
     ctx->decision_ready = false;
     ctx->last_projected_step = ctx->pending_step;
+    if (exch) ctx->swapped ^= 1;
     return host_out ? read_back(ctx, s, host_out) : GAC_OK;
 }
 
@@ -573,6 +585,12 @@ int gac_free(gac_ctx *ctx) {
 }
 
 const char *gac_last_error(const gac_ctx *ctx) { return ctx ? ctx->err : g_init_err; }
+
+int gac_next_gradient_set(const gac_ctx *ctx, int *set_out) {
+    if (!ctx || !set_out) return GAC_ERR_INVALID_ARG;
+    *set_out = ctx->swapped ? GAC_SET_D : GAC_SET_G;
+    return GAC_OK;
+}
 
 int gac_get_info(const gac_ctx *ctx, gac_info *out) {
     if (!ctx || !out) return GAC_ERR_INVALID_ARG;
@@ -658,6 +676,8 @@ extern "C" int gac_stats_static(const gac_tensor *list, uint32_t n, int g_dtype,
     if (pair_id(g_dtype, d_dtype) < 0)
         return fail(nullptr, GAC_ERR_DTYPE, "supported (g,d) element types: (f32,f32), (bf16,f32), (bf16,bf16)%s");
     if (int rc = check_hparams(hp)) return rc;
+    if (hp->state_mode == GAC_STATE_EXCHANGE)
+        return fail(nullptr, GAC_ERR_INVALID_ARG, "exchange mode needs a context (gac_init) to follow the buffer roles%s");
     if (cuda_device < 0 || cuda_device >= kMaxDevices)
         return fail(nullptr, GAC_ERR_INVALID_ARG, "cuda_device %s%lld out of range", "", cuda_device);
 

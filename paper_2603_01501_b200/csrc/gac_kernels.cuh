@@ -9,6 +9,8 @@
 #include <math.h>
 #include <stdint.h>
 
+#include <type_traits>
+
 #include "gac.h"
 
 namespace {
@@ -48,6 +50,7 @@ struct DevHP {
     unsigned staleness;
     int decide;      // 0: only publish the three sums (sharded form)
     double clip_max, clip_eps;
+    int swapped;     // exchange mode: 1 when the table's d addresses hold this step's gradient
 };
 
 struct F4 {
@@ -176,12 +179,18 @@ struct Elem<bf16_t> {
     }
 };
 
-__device__ __forceinline__ Chunk load_chunk(const Chunk *table, uint32_t c) {
+// swapped (exchange mode): the two address columns of the table trade roles.
+__device__ __forceinline__ Chunk load_chunk(const Chunk *table, uint32_t c, int swapped = 0) {
     const uint4 *p = reinterpret_cast<const uint4 *>(table + c);
     uint4 a = __ldg(p), b = __ldg(p + 1);
     Chunk ch;
     ch.g = (uint64_t(a.y) << 32) | a.x;
     ch.d = (uint64_t(a.w) << 32) | a.z;
+    if (swapped) {
+        const uint64_t t = ch.g;
+        ch.g = ch.d;
+        ch.d = t;
+    }
     ch.n = b.x;
     ch.flags = b.y;
     ch.pad = 0;
@@ -213,27 +222,7 @@ __device__ __forceinline__ double clip_factor(int regime, double dot, double gg,
 // Cosine with eps outside the root (App. A.1), the inclusive branches of
 // Algorithm 1, alpha = c_low/|c| (Eq. 5) or the caller's gain (Eq. 3), and the
 // multiplier of d in the rank-one form of App. A.2.
-__device__ void take_decision(double dot, double gg, double dd, const DevHP &hp, gac_result *r) {
-    if (hp.first_step) {   // Algorithm 1: g_0 = 0
-        dot = 0.0;
-        dd = 0.0;
-    }
-    r->dot = dot;
-    r->gg = gg;
-    r->dd = dd;
-    r->alpha = 1.0;
-    r->coef64 = 0.0;
-    r->coef = 0.0f;
-    r->out_norm = 0.0;
-    r->clip_scale = 1.0;
-    r->staleness = hp.staleness;
-    r->step = hp.step;
-    r->nonfinite = !(isfinite(dot) && isfinite(gg) && isfinite(dd));
-    if (r->nonfinite) {
-        r->cos = __longlong_as_double(0x7FF8000000000000LL);
-        r->regime = GAC_REGIME_VIOLATION;
-        return;
-    }
+__device__ void take_regime(double dot, double gg, double dd, const DevHP &hp, gac_result *r) {
     if (gg == 0.0 || dd == 0.0) {   // zero reference: u = 0, projector = identity
         r->cos = 0.0;
         r->regime = GAC_REGIME_SAFE;
@@ -262,6 +251,45 @@ __device__ void take_decision(double dot, double gg, double dd, const DevHP &hp,
     r->coef = __double2float_rn(k);
     r->clip_scale = clip_factor(r->regime, dot, gg, dd, hp.beta, double(r->coef), hp.clip_max, hp.clip_eps,
                                 &r->out_norm);
+}
+
+// The record of one step: the three sums, the zero reference of the first step
+// (Algorithm 1: g_0 = 0), the non-finite reading, the regime and gains, and --
+// for exchange mode -- which buffer set holds what the step sends on.
+__device__ void take_decision(double dot, double gg, double dd, const DevHP &hp, bool zero_reference,
+                              gac_result *r) {
+    if (zero_reference) {   // Algorithm 1: g_0 = 0
+        dot = 0.0;
+        dd = 0.0;
+    }
+    r->dot = dot;
+    r->gg = gg;
+    r->dd = dd;
+    r->alpha = 1.0;
+    r->coef64 = 0.0;
+    r->coef = 0.0f;
+    r->out_norm = 0.0;
+    r->clip_scale = 1.0;
+    r->staleness = hp.staleness;
+    r->step = hp.step;
+    r->g_set = uint32_t(hp.swapped);
+    r->out_set = r->g_set;
+    r->ref_lost = 0u;
+    r->reserved = 0u;
+    r->nonfinite = !(isfinite(dot) && isfinite(gg) && isfinite(dd));
+    if (r->nonfinite) {
+        r->cos = __longlong_as_double(0x7FF8000000000000LL);
+        r->regime = GAC_REGIME_VIOLATION;
+        return;
+    }
+    take_regime(dot, gg, dd, hp, r);
+    if (hp.state_mode == GAC_STATE_EXCHANGE) {
+        // exchange mode writes whatever differs from g into the buffers that held d
+        const bool writes = r->regime == GAC_REGIME_PROJECT ||
+                            (r->regime == GAC_REGIME_VIOLATION && hp.zero_on_violation) ||
+                            (r->regime == GAC_REGIME_SAFE && r->clip_scale != 1.0);
+        if (writes) r->out_set = r->g_set ^ 1u;
+    }
 }
 
 // ------------------------------------------------------------- stats kernel
@@ -370,12 +398,16 @@ gac_stats_kernel(const Chunk *__restrict__ chunks, uint32_t n_chunks, double *pa
     __shared__ double sm[T / 32][3];
     __shared__ bool is_last;
     double a_dot = 0.0, a_gg = 0.0, a_dd = 0.0;
-    if (hp.first_step) {
+    // Exchange mode after a non-finite step: the stored direction is gone, the
+    // step is taken against the zero reference like the first one.  Every CTA
+    // reads the flag here, before the last CTA can rewrite the record.
+    const bool zero_reference = hp.first_step || (hp.state_mode == GAC_STATE_EXCHANGE && rec->ref_lost);
+    if (zero_reference) {
         for (uint32_t c = blockIdx.x; c < n_chunks; c += gridDim.x)
-            stats_chunk<GT, false>(load_chunk(chunks, c), a_dot, a_gg, a_dd);
+            stats_chunk<GT, false>(load_chunk(chunks, c, hp.swapped), a_dot, a_gg, a_dd);
     } else {
         for (uint32_t c = blockIdx.x; c < n_chunks; c += gridDim.x)
-            stats_chunk<GT, true>(load_chunk(chunks, c), a_dot, a_gg, a_dd);
+            stats_chunk<GT, true>(load_chunk(chunks, c, hp.swapped), a_dot, a_gg, a_dd);
     }
     block_sum3<T>(a_dot, a_gg, a_dd, sm);
     if (threadIdx.x == 0) {
@@ -403,23 +435,23 @@ gac_stats_kernel(const Chunk *__restrict__ chunks, uint32_t n_chunks, double *pa
     if (threadIdx.x == 0) {
         *ticket = 0u;
         if (sums_out) {
-            sums_out[0] = hp.first_step ? 0.0 : s0;
+            sums_out[0] = zero_reference ? 0.0 : s0;
             sums_out[1] = s1;
-            sums_out[2] = hp.first_step ? 0.0 : s2;
+            sums_out[2] = zero_reference ? 0.0 : s2;
         }
-        if (hp.decide) take_decision(s0, s1, s2, hp, rec);
+        if (hp.decide) take_decision(s0, s1, s2, hp, zero_reference, rec);
     }
 }
 
 __global__ void gac_decide_kernel(const double *sums_in, gac_result *rec, DevHP hp) {
     if (threadIdx.x == 0 && blockIdx.x == 0)
-        take_decision(sums_in[0], sums_in[1], sums_in[2], hp, rec);
+        take_decision(sums_in[0], sums_in[1], sums_in[2], hp, hp.first_step != 0, rec);
 }
 
 // ----------------------------------------------------------- project kernel
 
 enum GOp { G_KEEP = 0, G_FMA = 1, G_ZERO = 2, G_SCALE = 3 };
-enum DOp { D_KEEP = 0, D_RAW = 1, D_NEW = 2 };
+enum DOp { D_KEEP = 0, D_RAW = 1, D_NEW = 2, D_OUT = 3 };   // D_OUT: the new g goes into d's buffer, g stays (exchange mode)
 
 template <bool BETA1>
 __device__ __forceinline__ float rank_one(float g, float d, float k, double beta, double s) {
@@ -434,6 +466,7 @@ template <typename GT, int GOP, int DOP, bool BETA1, int T, int U>
 __device__ __forceinline__ void project_chunk(const Chunk &ch, float k, double beta, double s) {
     void *g = reinterpret_cast<void *>(ch.g);
     void *d = reinterpret_cast<void *>(ch.d);
+    void *o = (DOP == D_OUT) ? d : g;   // where the outgoing gradient is stored
     const uint32_t tid = threadIdx.x;
     constexpr bool kReadG = (GOP == G_FMA) || (GOP == G_SCALE) || (DOP == D_RAW);
     constexpr bool kReadD = (GOP == G_FMA);
@@ -464,7 +497,7 @@ __device__ __forceinline__ void project_chunk(const Chunk &ch, float k, double b
                     out.w = rank_one<BETA1>(gv[u].w, dv[u].w, k, beta, s);
                 }
                 if (GOP == G_SCALE) out = F4{scaled(gv[u].x, s), scaled(gv[u].y, s), scaled(gv[u].z, s), scaled(gv[u].w, s)};
-                if (GOP != G_KEEP) Elem<GOf<GT>>::store4(g, v, out);
+                if (GOP != G_KEEP) Elem<GOf<GT>>::store4(o, v, out);
                 if (DOP == D_RAW) Elem<DOf<GT>>::store4(d, v, gv[u]);
                 if (DOP == D_NEW) {
                     if (GOP == G_FMA || GOP == G_SCALE) out = Elem<GOf<GT>>::template load4<GAC_LD_PROJECT>(g, v);   // the value as stored (rounded)
@@ -479,7 +512,7 @@ __device__ __forceinline__ void project_chunk(const Chunk &ch, float k, double b
             float out = (GOP == G_ZERO) ? 0.f : x;
             if (GOP == G_FMA) out = rank_one<BETA1>(x, Elem<DOf<GT>>::load1(d, i), k, beta, s);
             if (GOP == G_SCALE) out = scaled(x, s);
-            if (GOP != G_KEEP) Elem<GOf<GT>>::store1(g, i, out);
+            if (GOP != G_KEEP) Elem<GOf<GT>>::store1(o, i, out);
             if (DOP == D_RAW) Elem<DOf<GT>>::store1(d, i, x);
             if (DOP == D_NEW) {
                 if (GOP == G_FMA || GOP == G_SCALE) out = Elem<GOf<GT>>::load1(g, i);
@@ -492,7 +525,7 @@ __device__ __forceinline__ void project_chunk(const Chunk &ch, float k, double b
             float out = (GOP == G_ZERO) ? 0.f : x;
             if (GOP == G_FMA) out = rank_one<BETA1>(x, Elem<DOf<GT>>::load1(d, i), k, beta, s);
             if (GOP == G_SCALE) out = scaled(x, s);
-            if (GOP != G_KEEP) Elem<GOf<GT>>::store1(g, i, out);
+            if (GOP != G_KEEP) Elem<GOf<GT>>::store1(o, i, out);
             if (DOP == D_RAW) Elem<DOf<GT>>::store1(d, i, x);
             if (DOP == D_NEW) {
                 if (GOP == G_FMA || GOP == G_SCALE) out = Elem<GOf<GT>>::load1(g, i);
@@ -504,9 +537,9 @@ __device__ __forceinline__ void project_chunk(const Chunk &ch, float k, double b
 
 template <typename GT, int GOP, int DOP, bool BETA1>
 __device__ __forceinline__ void project_walk(const Chunk *chunks, uint32_t n_chunks, float k,
-                                             double beta, double s) {
+                                             double beta, double s, int swapped) {
     for (uint32_t c = blockIdx.x; c < n_chunks; c += gridDim.x)
-        project_chunk<GT, GOP, DOP, BETA1, ProjGeom<GT>::T, ProjGeom<GT>::U>(load_chunk(chunks, c), k, beta, s);
+        project_chunk<GT, GOP, DOP, BETA1, ProjGeom<GT>::T, ProjGeom<GT>::U>(load_chunk(chunks, c, swapped), k, beta, s);
 }
 
 // The regime is read from the device-resident record, so no host round trip
@@ -516,11 +549,17 @@ __device__ __forceinline__ void project_walk(const Chunk *chunks, uint32_t n_chu
 template <typename GT, int STATE, bool BETA1, bool ZERO>
 __global__ void __launch_bounds__(ProjGeom<GT>::T, ProjGeom<GT>::MINB)
 gac_project_kernel(const Chunk *__restrict__ chunks, uint32_t n_chunks, gac_result *rec,
-                   float coef_override, int use_override, double beta, double clip_max, double clip_eps) {
-    if (rec->nonfinite) return;   // reading taken for NaN/Inf: touch nothing
+                   float coef_override, int use_override, double beta, double clip_max, double clip_eps,
+                   int swapped) {
+    if (rec->nonfinite) {   // reading taken for NaN/Inf: touch nothing
+        // exchange mode: the roles swap all the same, so the stored direction is gone
+        if (STATE == GAC_STATE_EXCHANGE && blockIdx.x == 0 && threadIdx.x == 0) rec->ref_lost = 1u;
+        return;
+    }
     const int regime = rec->regime;
     const float k = use_override ? coef_override : rec->coef;
-    constexpr int dop = STATE == GAC_STATE_RAW ? D_RAW : (STATE == GAC_STATE_PROJECTED ? D_NEW : D_KEEP);
+    constexpr int dop = STATE == GAC_STATE_RAW ? D_RAW
+                        : (STATE == GAC_STATE_PROJECTED ? D_NEW : (STATE == GAC_STATE_EXCHANGE ? D_OUT : D_KEEP));
     double s = 1.0;
     if (clip_max > 0.0) {
         // recomputed here so that it belongs to the coefficient actually applied
@@ -532,16 +571,17 @@ gac_project_kernel(const Chunk *__restrict__ chunks, uint32_t n_chunks, gac_resu
         }
     }
     if (regime == GAC_REGIME_PROJECT) {
-        if (s != 1.0) project_walk<GT, G_FMA, dop, false>(chunks, n_chunks, k, beta, s);
-        else project_walk<GT, G_FMA, dop, BETA1>(chunks, n_chunks, k, beta, 1.0);
+        if (s != 1.0) project_walk<GT, G_FMA, dop, false>(chunks, n_chunks, k, beta, s, swapped);
+        else project_walk<GT, G_FMA, dop, BETA1>(chunks, n_chunks, k, beta, 1.0, swapped);
     } else if (ZERO && regime == GAC_REGIME_VIOLATION) {
-        project_walk<GT, G_ZERO, dop, true>(chunks, n_chunks, k, 1.0, 1.0);
+        project_walk<GT, G_ZERO, dop, true>(chunks, n_chunks, k, 1.0, 1.0, swapped);
     } else if (s != 1.0) {
-        project_walk<GT, G_SCALE, dop, true>(chunks, n_chunks, k, 1.0, s);   // safe step, clipped: g'' = s g
-    } else if (STATE != GAC_STATE_HOLD) {
+        project_walk<GT, G_SCALE, dop, true>(chunks, n_chunks, k, 1.0, s, swapped);   // safe step, clipped: g'' = s g
+    } else if (STATE != GAC_STATE_HOLD && STATE != GAC_STATE_EXCHANGE) {
         for (uint32_t c = blockIdx.x; c < n_chunks; c += gridDim.x)   // d' = g, g untouched
             project_chunk<GT, G_KEEP, D_RAW, true, ProjGeom<GT>::T, ProjGeom<GT>::UK>(load_chunk(chunks, c), k, 1.0, 1.0);
     }
+    // exchange mode, g unchanged: nothing to move -- the buffers that hold g become the stored direction
 }
 
 // ------------------------------------------------ projection fused with AdamW
@@ -604,7 +644,7 @@ __device__ __forceinline__ void adamw_elem(double g64, float &p, float &m, float
     v = __double2float_rn(v64);
 }
 
-template <typename GT, int GOP>
+template <typename GT, int GOP, bool STORE_D>
 __device__ __forceinline__ void adamw_chunk(const Chunk &ch, const OptChunk &oc, float k, double beta,
                                             double s, const AdamConst &a) {
     const void *g = reinterpret_cast<const void *>(ch.g);
@@ -644,7 +684,7 @@ __device__ __forceinline__ void adamw_chunk(const Chunk &ch, const OptChunk &oc,
                 for (int e = 0; e < 4; ++e) {
                     adamw_elem(outgoing64<GOP>(ge[e], de[e], k, beta, s), pe[e], me[e], ve[e], a);
                 }
-                Elem<DOf<GT>>::store4(d, w, gv[u]);                       // d' = g, the raw gradient
+                if (STORE_D) Elem<DOf<GT>>::store4(d, w, gv[u]);          // d' = g, the raw gradient
                 Elem<float>::store4(pp, w, F4{pe[0], pe[1], pe[2], pe[3]});
                 Elem<float>::store4(pm, w, F4{me[0], me[1], me[2], me[3]});
                 Elem<float>::store4(pv, w, F4{ve[0], ve[1], ve[2], ve[3]});
@@ -657,7 +697,7 @@ __device__ __forceinline__ void adamw_chunk(const Chunk &ch, const OptChunk &oc,
         const float dx = (GOP == G_FMA) ? Elem<DOf<GT>>::load1(d, i) : 0.f;
         float pe = Elem<float>::load1(pp, i), me = Elem<float>::load1(pm, i), ve = Elem<float>::load1(pv, i);
         adamw_elem(outgoing64<GOP>(x, dx, k, beta, s), pe, me, ve, a);
-        Elem<DOf<GT>>::store1(d, i, x);
+        if (STORE_D) Elem<DOf<GT>>::store1(d, i, x);
         Elem<float>::store1(pp, i, pe);
         Elem<float>::store1(pm, i, me);
         Elem<float>::store1(pv, i, ve);
@@ -680,12 +720,17 @@ __device__ __forceinline__ OptChunk load_opt_chunk(const OptChunk *table, uint32
 // applied updates lives in the decision record: every CTA reads it on entry,
 // and the last CTA to FINISH (arrival ticket, nobody waits) writes it back
 // incremented, so no CTA can see the new value during this launch.
-template <typename GT>
+// EXCH (exchange mode): d' = g costs nothing -- the buffers swap roles -- so no
+// state is stored and a skipped step moves no data at all.
+template <typename GT, bool EXCH>
 __global__ void __launch_bounds__(AdamGeom<GT>::T, AdamGeom<GT>::C)
 gac_adamw_kernel(const Chunk *__restrict__ chunks, const OptChunk *__restrict__ opt_chunks,
                  uint32_t n_chunks, gac_result *rec, unsigned *ticket, float coef_override,
-                 int use_override, double beta, double clip_max, double clip_eps, AdamDev o) {
-    if (rec->nonfinite) return;
+                 int use_override, double beta, double clip_max, double clip_eps, AdamDev o, int swapped) {
+    if (rec->nonfinite) {
+        if (EXCH && blockIdx.x == 0 && threadIdx.x == 0) rec->ref_lost = 1u;
+        return;
+    }
     const int regime = rec->regime;
     const float k = use_override ? coef_override : rec->coef;
     const unsigned long long t_prev = rec->applied_steps;
@@ -712,13 +757,13 @@ gac_adamw_kernel(const Chunk *__restrict__ chunks, const OptChunk *__restrict__ 
         a.eps = o.eps;
         a.lr_wd = o.lr * o.weight_decay;
         for (uint32_t c = blockIdx.x; c < n_chunks; c += gridDim.x) {
-            const Chunk ch = load_chunk(chunks, c);
+            const Chunk ch = load_chunk(chunks, c, swapped);
             const OptChunk oc = load_opt_chunk(opt_chunks, c);
-            if (regime == GAC_REGIME_PROJECT) adamw_chunk<GT, G_FMA>(ch, oc, k, beta, s, a);
-            else if (s != 1.0) adamw_chunk<GT, G_SCALE>(ch, oc, k, 1.0, s, a);
-            else adamw_chunk<GT, G_KEEP>(ch, oc, k, 1.0, 1.0, a);
+            if (regime == GAC_REGIME_PROJECT) adamw_chunk<GT, G_FMA, !EXCH>(ch, oc, k, beta, s, a);
+            else if (s != 1.0) adamw_chunk<GT, G_SCALE, !EXCH>(ch, oc, k, 1.0, s, a);
+            else adamw_chunk<GT, G_KEEP, !EXCH>(ch, oc, k, 1.0, 1.0, a);
         }
-    } else {
+    } else if (!EXCH) {
         for (uint32_t c = blockIdx.x; c < n_chunks; c += gridDim.x)   // skipped step: d' = g only
             project_chunk<GT, G_KEEP, D_RAW, true, AdamGeom<GT>::T, AdamGeom<GT>::U>(load_chunk(chunks, c), k, 1.0, 1.0);
     }
@@ -734,17 +779,29 @@ gac_adamw_kernel(const Chunk *__restrict__ chunks, const OptChunk *__restrict__ 
     }
 }
 
-using ProjectKernel = void (*)(const Chunk *, uint32_t, gac_result *, float, int, double, double, double);
+using ProjectKernel = void (*)(const Chunk *, uint32_t, gac_result *, float, int, double, double, double, int);
 
 template <typename GT, int STATE>
 ProjectKernel pick_project(bool beta1, bool zero) {
     if (beta1) return zero ? gac_project_kernel<GT, STATE, true, true> : gac_project_kernel<GT, STATE, true, false>;
     return zero ? gac_project_kernel<GT, STATE, false, true> : gac_project_kernel<GT, STATE, false, false>;
 }
+// Exchange mode stores g' with g's element type into d's buffers: only pairs of one type have it.
+template <typename GT>
+using SameTypes = std::integral_constant<bool, std::is_same<GOf<GT>, DOf<GT>>::value>;
+template <typename GT>
+ProjectKernel pick_exchange(bool beta1, bool zero, std::true_type) {
+    return pick_project<GT, GAC_STATE_EXCHANGE>(beta1, zero);
+}
+template <typename GT>
+ProjectKernel pick_exchange(bool, bool, std::false_type) {
+    return nullptr;
+}
 template <typename GT>
 ProjectKernel pick_project(int state, bool beta1, bool zero) {
     if (state == GAC_STATE_RAW) return pick_project<GT, GAC_STATE_RAW>(beta1, zero);
     if (state == GAC_STATE_PROJECTED) return pick_project<GT, GAC_STATE_PROJECTED>(beta1, zero);
+    if (state == GAC_STATE_EXCHANGE) return pick_exchange<GT>(beta1, zero, SameTypes<GT>{});
     return pick_project<GT, GAC_STATE_HOLD>(beta1, zero);
 }
 

@@ -92,7 +92,11 @@ def test_argument_errors_need_no_device(lib):
     assert _init(lib, [ok], eps=-1.0)[0] == gb.GAC_ERR_INVALID_ARG
     assert _init(lib, [ok], beta=float("nan"))[0] == gb.GAC_ERR_INVALID_ARG
     assert _init(lib, [ok], mode=5)[0] == gb.GAC_ERR_INVALID_ARG
-    assert _init(lib, [ok], state_mode=3)[0] == gb.GAC_ERR_INVALID_ARG
+    assert _init(lib, [ok], state_mode=4)[0] == gb.GAC_ERR_INVALID_ARG
+    # exchange mode swaps the roles of the two buffer sets: one element type for both
+    rc, msg = _init(lib, [ok], g_dt=1, d_dt=0, state_mode=gb.GAC_STATE_EXCHANGE)
+    assert rc == gb.GAC_ERR_DTYPE and "exchange" in msg
+    assert _init(lib, [ok], state_mode=gb.GAC_STATE_EXCHANGE)[0] in (gb.GAC_OK, gb.GAC_ERR_CUDA)
     assert _init(lib, [ok], mode=1, alpha_fixed=-1.0)[0] == gb.GAC_ERR_INVALID_ARG
     assert _init(lib, [ok], reserved=1)[0] == gb.GAC_ERR_INVALID_ARG
     assert _init(lib, [(4097, 8192, 16)])[0] == gb.GAC_ERR_INVALID_ARG       # not element-aligned
@@ -116,6 +120,7 @@ def test_null_context_is_rejected(lib):
     assert lib.gac_stats_partial(None, 1, 0, None, None) == gb.GAC_ERR_INVALID_ARG
     assert lib.gac_decide(None, None, None, None) == gb.GAC_ERR_INVALID_ARG
     assert lib.gac_set_launch(None, 0, 0) == gb.GAC_ERR_INVALID_ARG
+    assert lib.gac_next_gradient_set(None, None) == gb.GAC_ERR_INVALID_ARG
     assert lib.gac_free(None) == gb.GAC_OK
     assert lib.gac_last_error(None) is not None
 

@@ -1,0 +1,280 @@
+"""GPU parity of exchange mode (state_mode EXCHANGE) against the CPU oracle.
+
+Exchange mode computes what the paper's rule computes -- g' from Eq. 5 and the
+stored direction d' = g of App. A.2 -- without the copy that refreshes the
+snapshot: the buffers that held g become the stored direction, g' (when it
+differs from g) lands in the buffers that held d, and the two sets swap roles
+after every step.  The oracle therefore runs the plain RAW rule; the tests map
+its g' and d' onto the buffer sets the record names and check, bit for bit,
+that nothing else was written.
+"""
+import dataclasses
+import math
+
+import pytest
+import torch
+
+from oracle import gac_oracle as orc
+from paper_2603_01501_b200 import binding as gb
+from paper_2603_01501_b200 import synth
+
+from gpu_util import check_decision, check_sums, max_ulp, ordered_int, to_orc_hp
+
+pytestmark = pytest.mark.gpu
+
+BITS = {torch.float32: torch.int32, torch.bfloat16: torch.int16}
+
+
+def raw_hp(hp: gb.HParams) -> orc.HParams:
+    """The oracle's rule for an exchange-mode context: the paper's RAW state."""
+    return to_orc_hp(dataclasses.replace(hp, state_mode=gb.GAC_STATE_RAW))
+
+
+def same_bits(a: torch.Tensor, b: torch.Tensor) -> bool:
+    return torch.equal(a.cpu().view(BITS[a.dtype]), b.cpu().view(BITS[b.dtype]))
+
+
+def ar_gradients(shapes, sig, rhos, dtype, seed):
+    """One gradient list per entry of rhos: cosine about rho to the previous one (None = fresh noise)."""
+    gen = torch.Generator().manual_seed(seed)
+    prev = None
+    for rho in rhos:
+        noise = [torch.randn(n, generator=gen) * s for (_, n), s in zip(shapes, sig)]
+        if rho is None or prev is None:
+            g = noise
+        else:
+            g = [rho * a + math.sqrt(1 - rho * rho) * b for a, b in zip(prev, noise)]
+        g = [x.to(dtype) for x in g]
+        prev = [x.float().clone() for x in g]      # the caller may plant a NaN in what it gets
+        yield g
+
+
+def run_exchange_sequence(dtype, hp, rhos, shapes_name="mini", nan_at=(), views=False):
+    """Steps a context in exchange mode and the RAW oracle side by side.  Returns the regimes met."""
+    shapes = synth.decoder_tensor_list(synth.DIMS[shapes_name])
+    sig = synth.per_tensor_scales(2, len(shapes))
+    pad = 3 if views else 0     # odd element offsets: the element-wise path
+    bufs = [[torch.full((n + 2 * pad + 1,), 5.0, dtype=dtype, device="cuda") for _, n in shapes] for _ in range(2)]
+    sets = [[b[pad:pad + n] if views else b[:n] for b, (_, n) in zip(bs, shapes)] for bs in bufs]
+    for t in sets[1]:
+        t.fill_(float("nan"))                      # never read on step 1
+    ctx = gb.gac_init(sets[0], sets[1], hp)
+    if views:
+        assert gb.gac_get_info(ctx).misaligned_tensors == len(shapes)
+    ohp = raw_hp(hp)
+    d_ref = [torch.full((n,), float("nan"), dtype=dtype) for _, n in shapes]
+    regimes, lost = [], False
+    for t, g in enumerate(ar_gradients(shapes, sig, rhos, dtype, seed=11), start=1):
+        if t in nan_at:
+            g[len(g) // 2][7] = float("nan")
+        gi = gb.gac_next_gradient_set(ctx)
+        assert gi == (t - 1) % 2                    # the roles alternate, whatever the steps decide
+        di = gi ^ 1
+        for dst, src in zip(sets[gi], g):
+            dst.copy_(src)
+        before_d = [x.clone() for x in sets[di]]
+        first = (t == 1) or lost                    # zero reference: Algorithm 1's g_0, or a lost direction
+        g_ref = [x.clone() for x in g]
+        dec = orc.decide(orc.stats(g_ref, d_ref, first_step=first), ohp, first)
+        res = gb.gac_stats(ctx, t)
+        after = gb.gac_project(ctx, coef_override=dec.coef if dec.regime == orc.PROJECT else None, fetch=True)
+        torch.cuda.synchronize()
+        check_sums(res, dec)
+        assert res.g_set == gi and after.g_set == gi
+        # the buffers that held g are never written: they are the stored direction now
+        for a, b in zip(sets[gi], g):
+            assert same_bits(a, b), f"step {t}: the gradient buffers were modified"
+        if dec.nonfinite:
+            assert res.nonfinite == 1 and after.ref_lost == 1 and after.out_set == gi
+            for a, b in zip(sets[di], before_d):
+                assert same_bits(a, b)
+            lost = True
+            regimes.append("nonfinite")
+            continue
+        lost = False
+        check_decision(res, dec)
+        assert after.ref_lost == 0
+        orc.project(g_ref, d_ref, ohp, dec, first_step=first)      # g_ref <- g', d_ref <- raw g
+        changed = (dec.regime == orc.PROJECT or (dec.regime == orc.VIOLATION and hp.zero_on_violation)
+                   or (dec.regime == orc.SAFE and dec.clip_scale != 1.0))
+        assert after.out_set == (di if changed else gi)
+        lim = 4 if dtype == torch.float32 else 1
+        for i, (a, b) in enumerate(zip(sets[after.out_set], g_ref)):
+            assert max_ulp(a.cpu(), b) <= lim, f"step {t} tensor {i}: outgoing gradient off by {max_ulp(a.cpu(), b)} ulp"
+        if not changed:
+            for a, b in zip(sets[di], before_d):
+                assert same_bits(a, b), f"step {t}: a step that leaves g alone must not write anything"
+        for a, b in zip(sets[gi], d_ref):
+            assert same_bits(a, b)                  # stored direction = raw gradient, bit for bit
+        regimes.append(dec.regime)
+    if views:                                       # nothing outside the views was touched
+        for bs in bufs:
+            for b, (_, n) in zip(bs, shapes):
+                assert bool((b[:pad] == 5.0).all()) and bool((b[pad + n:] == 5.0).all())
+    gb.gac_free(ctx)
+    return regimes
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16], ids=["f32", "bf16"])
+def test_exchange_mode_over_all_regimes(dtype):
+    regimes = run_exchange_sequence(dtype, gb.HParams(state_mode=gb.GAC_STATE_EXCHANGE),
+                                    rhos=(None, 0.0, 0.15, 0.8, 0.02, 0.2, 0.25))
+    assert set(regimes) == {orc.SAFE, orc.PROJECT, orc.VIOLATION}
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16], ids=["f32", "bf16"])
+def test_exchange_mode_restarts_after_a_nonfinite_step(dtype):
+    regimes = run_exchange_sequence(dtype, gb.HParams(state_mode=gb.GAC_STATE_EXCHANGE),
+                                    rhos=(None, 0.2, 0.2, 0.2, 0.2, 0.9), nan_at=(3,))
+    # step 3 is reported and writes nothing; step 4 is taken against the zero reference (safe)
+    assert regimes[2] == "nonfinite" and regimes[3] == orc.SAFE and regimes[4] == orc.PROJECT
+
+
+@pytest.mark.parametrize("hp", [
+    gb.HParams(state_mode=gb.GAC_STATE_EXCHANGE, zero_on_violation=1),
+    gb.HParams(state_mode=gb.GAC_STATE_EXCHANGE, clip_max_norm=1e-3),
+    gb.HParams(state_mode=gb.GAC_STATE_EXCHANGE, clip_max_norm=1e6),
+    gb.HParams(state_mode=gb.GAC_STATE_EXCHANGE, mode=gb.GAC_MODE_FIXED, alpha_fixed=0.25, beta=1.5),
+    gb.HParams(state_mode=gb.GAC_STATE_EXCHANGE, mode=gb.GAC_MODE_FIXED, alpha_fixed=0.0),
+], ids=["zero_on_violation", "clipped", "clip_inactive", "fixed_gains", "full_projection"])
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16], ids=["f32", "bf16"])
+def test_exchange_mode_variants(hp, dtype):
+    run_exchange_sequence(dtype, hp, rhos=(None, 0.0, 0.15, 0.8, 0.02, 0.2))
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16], ids=["f32", "bf16"])
+def test_exchange_mode_on_unaligned_views_and_a_larger_list(dtype):
+    hp = gb.HParams(state_mode=gb.GAC_STATE_EXCHANGE, c_low=0.05, c_high=0.6)
+    run_exchange_sequence(dtype, hp, rhos=(None, 0.3, 0.01, 0.9), views=True)
+    run_exchange_sequence(dtype, hp, rhos=(None, 0.3, 0.5), shapes_name="small")
+
+
+@pytest.mark.parametrize("n", [1, 3, 4, 5, 1023, 4097, 16385, 5 * 16384 + 7])
+def test_exchange_mode_sizes_and_tails(n):
+    gen = torch.Generator().manual_seed(n)
+    d = torch.randn(n, generator=gen)
+    g = 0.5 * d + math.sqrt(0.75) * torch.randn(n, generator=gen)
+    hp = gb.HParams(state_mode=gb.GAC_STATE_EXCHANGE, c_low=0.05, c_high=2.0)
+    a, b = [g.cuda()], [d.cuda()]
+    ctx = gb.gac_init(a, b, hp)
+    g_ref, d_ref = [g.clone()], [d.clone()]
+    dec = orc.step(g_ref, d_ref, raw_hp(hp))
+    res = gb.gac_stats(ctx, 2)
+    after = gb.gac_project(ctx, coef_override=dec.coef if dec.regime == orc.PROJECT else None, fetch=True)
+    check_sums(res, dec)
+    check_decision(res, dec)
+    if dec.regime == orc.PROJECT:
+        assert after.out_set == gb.GAC_SET_D
+        assert max_ulp(b[0].cpu(), g_ref[0]) <= 4
+    assert same_bits(a[0], g) and gb.gac_next_gradient_set(ctx) == gb.GAC_SET_D
+    gb.gac_free(ctx)
+
+
+def test_exchange_mode_sharded_form_and_rebind():
+    """Local sums, the caller's reduction, the decision, the projection: the same roles and
+    results as the unsharded calls; gac_rebind starts the alternation over."""
+    shapes = synth.decoder_tensor_list(synth.DIMS["mini"])
+    g, d = synth.gradient_list(shapes, 0.4, config_id=2, device="cuda")
+    g_cpu, d_cpu = [t.cpu() for t in g], [t.cpu() for t in d]
+    hp = gb.HParams(state_mode=gb.GAC_STATE_EXCHANGE, c_low=0.05, c_high=0.9)
+    ctx = gb.gac_init(g, d, hp)
+    sums = torch.zeros(3, dtype=torch.float64, device="cuda")
+    gb.gac_stats_partial(ctx, 2, sums)
+    res = gb.gac_decide(ctx, sums)
+    g_ref, d_ref = [t.clone() for t in g_cpu], [t.clone() for t in d_cpu]
+    dec = orc.step(g_ref, d_ref, raw_hp(hp))
+    after = gb.gac_project(ctx, coef_override=dec.coef, fetch=True)
+    check_sums(res, dec)
+    check_decision(res, dec)
+    assert dec.regime == orc.PROJECT and after.out_set == gb.GAC_SET_D
+    assert all(max_ulp(a.cpu(), b) <= 4 for a, b in zip(d, g_ref))
+    assert all(same_bits(a, b) for a, b in zip(g, g_cpu))
+    assert gb.gac_next_gradient_set(ctx) == gb.GAC_SET_D
+    # second step with swapped roles through the sharded calls: d holds the gradient, g the direction
+    g2 = [0.3 * a + math.sqrt(1 - 0.09) * torch.randn_like(a) * a.std() for a in g_cpu]
+    for dst, src in zip(d, g2):
+        dst.copy_(src)
+    gb.gac_stats_partial(ctx, 3, sums)
+    res = gb.gac_decide(ctx, sums)
+    g_ref2 = [t.clone() for t in g2]
+    dec = orc.step(g_ref2, d_ref, raw_hp(hp))
+    after = gb.gac_project(ctx, coef_override=dec.coef if dec.regime == orc.PROJECT else None, fetch=True)
+    check_sums(res, dec)
+    check_decision(res, dec)
+    assert res.g_set == gb.GAC_SET_D and dec.regime == orc.PROJECT and after.out_set == gb.GAC_SET_G
+    assert all(max_ulp(a.cpu(), b) <= 4 for a, b in zip(g, g_ref2))
+    assert gb.gac_next_gradient_set(ctx) == gb.GAC_SET_G
+    gb.gac_stats(ctx, 4, fetch=False)
+    gb.gac_project(ctx)
+    assert gb.gac_next_gradient_set(ctx) == gb.GAC_SET_D
+    gb.gac_rebind(ctx, g, d)
+    assert gb.gac_next_gradient_set(ctx) == gb.GAC_SET_G
+    gb.gac_free(ctx)
+
+
+def test_exchange_mode_needs_one_element_type_and_a_context():
+    g = [torch.ones(64, dtype=torch.bfloat16, device="cuda")]
+    d = [torch.ones(64, device="cuda")]
+    hp = gb.HParams(state_mode=gb.GAC_STATE_EXCHANGE)
+    with pytest.raises(gb.GacError) as e:
+        gb.gac_init(g, d, hp)
+    assert e.value.status == gb.GAC_ERR_DTYPE
+    import ctypes
+    out = torch.zeros(ctypes.sizeof(gb.gac_result), dtype=torch.uint8, device="cuda")
+    with pytest.raises(gb.GacError) as e:
+        gb.gac_stats_static(d, [torch.ones(64, device="cuda")], hp, 2, out)
+    assert e.value.status == gb.GAC_ERR_INVALID_ARG
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16], ids=["f32", "bf16"])
+def test_exchange_mode_fused_adamw(dtype):
+    """The fused optimizer step in exchange mode: same p, m, v as the oracle's AdamW on the RAW
+    rule's g', and neither buffer set is written at all."""
+    shapes = synth.decoder_tensor_list(synth.DIMS["mini"])
+    sig = synth.per_tensor_scales(2, len(shapes))
+    gen = torch.Generator().manual_seed(7)
+    p_cpu = [torch.randn(n, generator=gen) * 0.02 for _, n in shapes]
+    m_cpu = [torch.zeros(n) for _, n in shapes]
+    v_cpu = [torch.zeros(n) for _, n in shapes]
+    sets = [[torch.full((n,), float("nan"), dtype=dtype, device="cuda") for _, n in shapes] for _ in range(2)]
+    p_gpu, m_gpu, v_gpu = ([t.cuda() for t in l] for l in (p_cpu, m_cpu, v_cpu))
+    hp = gb.HParams(state_mode=gb.GAC_STATE_EXCHANGE, clip_max_norm=0.5)
+    ctx = gb.gac_init(sets[0], sets[1], hp)
+    gb.gac_attach_adamw(ctx, p_gpu, m_gpu, v_gpu, applied_steps=0)
+    gopt, oopt = gb.AdamW(lr=1e-3), orc.AdamW(lr=1e-3)
+    ohp = raw_hp(hp)
+    d_ref = [torch.full((n,), float("nan"), dtype=dtype) for _, n in shapes]
+    applied, regimes = 0, []
+    for t, g in enumerate(ar_gradients(shapes, sig, (None, 0.0, 0.3, 0.9, 0.2, 0.01, 0.5), dtype, seed=3), start=1):
+        gi = gb.gac_next_gradient_set(ctx)
+        assert gi == (t - 1) % 2
+        for dst, src in zip(sets[gi], g):
+            dst.copy_(src)
+        before_d = [x.clone() for x in sets[gi ^ 1]]
+        first = t == 1
+        dec = orc.decide(orc.stats(g, d_ref, first_step=first), ohp, first)
+        m_before = [x.clone() for x in m_cpu]
+        d_before = [x.clone().float() for x in d_ref]
+        applied += int(orc.project_adamw(g, d_ref, p_cpu, m_cpu, v_cpu, ohp, dec, oopt, applied + 1, first))
+        res = gb.gac_stats(ctx, t)
+        after = gb.gac_project_adamw(ctx, gopt, coef_override=dec.coef if dec.regime == orc.PROJECT else None,
+                                     fetch=True)
+        check_sums(res, dec)
+        check_decision(res, dec)
+        assert after.applied_steps == applied
+        for i in range(len(shapes)):
+            assert same_bits(sets[gi][i], g[i]) and same_bits(sets[gi][i], d_ref[i])
+            assert same_bits(sets[gi ^ 1][i], before_d[i]), "exchange mode stores no state"
+            gmag = g[i].float().abs() + abs(dec.coef) * d_before[i].abs().nan_to_num(0.0)
+            for name, a, b, slack in (("v", v_gpu[i], v_cpu[i], None),
+                                      ("m", m_gpu[i], m_cpu[i], 1e-13 * (m_before[i].abs() + gmag)),
+                                      ("p", p_gpu[i], p_cpu[i], torch.full_like(p_cpu[i], 1e-10 * oopt.lr))):
+                a_cpu = a.cpu()
+                ok = (ordered_int(a_cpu) - ordered_int(b)).abs() <= 4
+                if slack is not None:
+                    ok |= (a_cpu.double() - b.double()).abs() <= slack.double()
+                assert bool(ok.all()), f"step {t} tensor {i} {name}"
+                a.copy_(b)       # every step is compared from identical state
+        regimes.append(dec.regime)
+    assert set(regimes) == {0, 1, 2}
+    gb.gac_free(ctx)
