@@ -243,6 +243,52 @@ def time_unchanged_regime(wl: Workload, steps: int):
             "hbm_gbs": nbytes / (ms * 1e-3) / 1e9}
 
 
+def time_exchange_mode(wl: Workload, steps: int):
+    """The same list in exchange mode (g and d of one element type): the stored
+    direction is refreshed by swapping the roles of the two buffer sets, so a
+    projection step reads g and d and writes g' once -- (sg+sd) + (sg+sd+sg)
+    bytes per parameter -- and a step that leaves g alone moves only the (sg+sd)
+    of the reduction.  Every step's gradient is written into the set that is free."""
+    gb = wl.gb
+    if wl.g_dtype != wl.d_dtype:
+        return {"skipped": "exchange mode needs g and d of one element type"}
+    sets = [wl.g, wl.d]
+    sg = 2 if wl.g_dtype == torch.bfloat16 else 4
+    out = {}
+    for label, thr in (("project", FORCE), ("unchanged", {})):
+        ctx = gb.gac_init(sets[0], sets[1], gb.HParams(state_mode=gb.GAC_STATE_EXCHANGE, **thr))
+        step_no, evs = 1, []
+        for i in range(3 + steps):
+            gi = gb.gac_next_gradient_set(ctx)
+            synth.refresh_gradient_list(sets[gi], sets[gi ^ 1], wl.sigma, wl.rho, wl.gen, wl.scratch)
+            step_no += 1
+            e = [torch.cuda.Event(enable_timing=True) for _ in range(3)]
+            e[0].record()
+            gb.gac_stats(ctx, step_no, fetch=False)
+            e[1].record()
+            gb.gac_project(ctx)
+            e[2].record()
+            if i >= 3:
+                evs.append(e)
+        gi = gb.gac_next_gradient_set(ctx)
+        synth.refresh_gradient_list(sets[gi], sets[gi ^ 1], wl.sigma, wl.rho, wl.gen, wl.scratch)
+        res = gb.gac_stats(ctx, step_no + 1)
+        gb.gac_project(ctx)
+        torch.cuda.synchronize()
+        gb.gac_free(ctx)
+        s_ms = sum(a.elapsed_time(b) for a, b, _ in evs) / len(evs)
+        p_ms = sum(b.elapsed_time(c) for _, b, c in evs) / len(evs)
+        proj_bpp = 3 * sg if label == "project" else 0
+        out[label] = {"regime": gb.REGIME_NAMES[res.regime], "cos": res.cos, "ms_per_step": s_ms + p_ms,
+                      "stats_ms": s_ms, "project_ms": p_ms, "value": wl.params / ((s_ms + p_ms) * 1e-3),
+                      "unit": UNIT, "bytes_per_param": 2 * sg + proj_bpp,
+                      "hbm_gbs": wl.params * (2 * sg + proj_bpp) / ((s_ms + p_ms) * 1e-3) / 1e9,
+                      "project_kernel_gbs": (wl.params * proj_bpp / (p_ms * 1e-3) / 1e9) if proj_bpp else None}
+    # leave the workload as it was found: wl.g holds a gradient, wl.d its stored direction
+    synth.refresh_gradient_list(wl.g, wl.d, wl.sigma, wl.rho, wl.gen, wl.scratch)
+    return out
+
+
 def time_fused_adamw(wl: Workload, steps: int):
     """stats + the projection fused with AdamW (Table 2 values): the update goes
     straight into p, m, v and g' is never written.  Moves (sg+4) + (sg+4+12) read
@@ -552,6 +598,8 @@ def main():
         line["unchanged_regime"] = time_unchanged_regime(wl, min(args.steps, 10))
     if world == 1 and args.adamw:
         line["fused_adamw"] = time_fused_adamw(wl, min(args.steps, 10))
+    if world == 1 and wl.g_dtype == wl.d_dtype:
+        line["exchange_mode"] = time_exchange_mode(wl, min(args.steps, 10))
     if not args.no_e2e:
         # every rank takes the same branch: the decision to run is agreed on first, and the
         # result is reduced by all ranks whether or not a rank failed
@@ -591,6 +639,8 @@ def main():
                          "params": wl2.params, "steps": min(args.steps, 10),
                          "value": wl2.params / (also["ms_per_step"] * 1e-3), "unit": UNIT,
                          "regime_check": {"cos": r2.cos, "regime": gb.REGIME_NAMES[r2.regime]}})
+            if wl2.g_dtype == wl2.d_dtype:
+                also["exchange_mode"] = time_exchange_mode(wl2, min(args.steps, 10))
             line["also"] = also
             wl2.close()
         else:

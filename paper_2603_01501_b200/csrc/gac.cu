@@ -230,7 +230,10 @@ int build_table(gac_ctx *c) {
     c->n_chunks = table.size();
 
     c->threads_stats = stats_threads_of(c->pair);
-    c->threads_project = with_pair(c->pair, [](auto tag) { return ProjGeom<decltype(tag)>::T; });
+    const bool exch = (c->hp.state_mode == GAC_STATE_EXCHANGE);
+    c->threads_project = with_pair(c->pair, [exch](auto tag) {
+        return exch ? ExchGeom<decltype(tag)>::T : ProjGeom<decltype(tag)>::T;
+    });
     int occ_s = resident_ctas(stats_kernel_of(c->pair), c->threads_stats);
     const bool beta1 = (c->hp.beta == 1.0), zero = (c->hp.zero_on_violation != 0);
     const int state_mode = c->hp.state_mode;
@@ -241,7 +244,9 @@ int build_table(gac_ctx *c) {
     c->project_fn = reinterpret_cast<const void *>(pk);
     int occ_p = resident_ctas(pk, c->threads_project);
     const int cap_s = stats_cap_of(c->pair);
-    const int cap_p = with_pair(c->pair, [](auto tag) { return ProjGeom<decltype(tag)>::C; });
+    const int cap_p = with_pair(c->pair, [exch](auto tag) {
+        return exch ? ExchGeom<decltype(tag)>::C : ProjGeom<decltype(tag)>::C;
+    });
     if (cap_s > 0) occ_s = std::min(occ_s, cap_s);
     if (cap_p > 0) occ_p = std::min(occ_p, cap_p);
     if (c->ctas_per_sm > 0) {

@@ -138,6 +138,8 @@ struct StatsGeom;   // fused triple reduction
 template <typename P>
 struct ProjGeom;    // projection + state refresh
 template <typename P>
+struct ExchGeom;    // projection in exchange mode (two reads, one write per element)
+template <typename P>
 struct AdamGeom;    // projection fused with AdamW
 #ifdef GAC_GEOMETRY_HEADER
 #include GAC_GEOMETRY_HEADER
@@ -148,6 +150,9 @@ template <> struct StatsGeom<bf16_pair_t> { static constexpr int T = 256, U = 8,
 template <> struct ProjGeom<float>        { static constexpr int T = 256, U = 8, UK = 16, C = 1, MINB = 1; };
 template <> struct ProjGeom<bf16_t>       { static constexpr int T = 512, U = 4, UK = 8, C = 1, MINB = 1; };
 template <> struct ProjGeom<bf16_pair_t>  { static constexpr int T = 512, U = 8, UK = 8, C = 1, MINB = 1; };
+template <> struct ExchGeom<float>        { static constexpr int T = 512, U = 4, UK = 8, C = 1, MINB = 1; };
+template <> struct ExchGeom<bf16_t>       { static constexpr int T = 512, U = 4, UK = 8, C = 1, MINB = 1; };   // pair not served
+template <> struct ExchGeom<bf16_pair_t>  { static constexpr int T = 512, U = 4, UK = 8, C = 2, MINB = 2; };
 template <> struct AdamGeom<float>        { static constexpr int T = 1024, U = 1, C = 1; };
 template <> struct AdamGeom<bf16_t>       { static constexpr int T = 1024, U = 1, C = 1; };
 template <> struct AdamGeom<bf16_pair_t>  { static constexpr int T = 1024, U = 1, C = 1; };
@@ -535,11 +540,16 @@ __device__ __forceinline__ void project_chunk(const Chunk &ch, float k, double b
     }
 }
 
+// Geometry of the projection kernel for a state mode.
+template <typename GT, int STATE>
+using ProjGeomOf = typename std::conditional<STATE == GAC_STATE_EXCHANGE, ExchGeom<GT>, ProjGeom<GT>>::type;
+
 template <typename GT, int GOP, int DOP, bool BETA1>
 __device__ __forceinline__ void project_walk(const Chunk *chunks, uint32_t n_chunks, float k,
                                              double beta, double s, int swapped) {
+    using Geom = typename std::conditional<DOP == D_OUT, ExchGeom<GT>, ProjGeom<GT>>::type;
     for (uint32_t c = blockIdx.x; c < n_chunks; c += gridDim.x)
-        project_chunk<GT, GOP, DOP, BETA1, ProjGeom<GT>::T, ProjGeom<GT>::U>(load_chunk(chunks, c, swapped), k, beta, s);
+        project_chunk<GT, GOP, DOP, BETA1, Geom::T, Geom::U>(load_chunk(chunks, c, swapped), k, beta, s);
 }
 
 // The regime is read from the device-resident record, so no host round trip
@@ -547,7 +557,7 @@ __device__ __forceinline__ void project_walk(const Chunk *chunks, uint32_t n_chu
 // the host already knows (state mode, beta == 1, zero_on_violation) is fixed at
 // compile time so that each instantiation holds only the loops it can reach.
 template <typename GT, int STATE, bool BETA1, bool ZERO>
-__global__ void __launch_bounds__(ProjGeom<GT>::T, ProjGeom<GT>::MINB)
+__global__ void __launch_bounds__((ProjGeomOf<GT, STATE>::T), (ProjGeomOf<GT, STATE>::MINB))
 gac_project_kernel(const Chunk *__restrict__ chunks, uint32_t n_chunks, gac_result *rec,
                    float coef_override, int use_override, double beta, double clip_max, double clip_eps,
                    int swapped) {

@@ -50,3 +50,50 @@ def test_controller_follows_algorithm_1_on_autograd_gradients():
     state = ctl.state_dict()
     assert state["t"] == len(order)
     ctl.close()
+
+
+def test_controller_in_exchange_mode_matches_the_raw_rule():
+    """Same loop with exchange=True: the snapshot is refreshed by swapping tensors, `.grad`
+    follows the outgoing gradient, and the values are those of the paper's rule."""
+    torch.manual_seed(0)
+    net = torch.nn.Sequential(torch.nn.Linear(37, 129), torch.nn.Tanh(), torch.nn.Linear(129, 5)).cuda()
+    hp = gb.HParams(c_low=0.05, c_high=0.9)
+    ctl = GradientAlignmentController(net.parameters(), hp, exchange=True)
+    opt = torch.optim.SGD(net.parameters(), lr=1e-3)
+    ohp = to_orc_hp(hp)                      # the oracle runs the RAW rule
+    d_ref = None
+    batches = [torch.randn(64, 37, device="cuda") for _ in range(3)]
+    targets = [torch.randn(64, 5, device="cuda") for _ in range(3)]
+    seen = set()
+    for t, b in enumerate([0, 0, 1, 1, 1, 2, 0], start=1):
+        if t == 1:
+            opt.zero_grad(set_to_none=True)
+        else:
+            ctl.zero_grad()
+        loss = torch.nn.functional.mse_loss(net(batches[b]), targets[b])
+        loss.backward()
+        raw = [p.grad.detach().view(-1).cpu().clone() for p in net.parameters()]
+        g_ref = [x.clone() for x in raw]
+        if d_ref is None:
+            d_ref = [torch.zeros_like(x) for x in g_ref]
+        dec = orc.step(g_ref, d_ref, ohp, first_step=(t == 1))
+        take = ctl.step()
+        res = ctl.last
+        check_sums(res, dec)
+        check_decision(res, dec)
+        assert take == (dec.regime != orc.VIOLATION)
+        for p, want, snap, r in zip(net.parameters(), g_ref, ctl.snapshot, raw):
+            assert torch.equal(snap.cpu(), r)                       # stored direction = raw gradient
+            tol = 2e-7 * float(want.abs().max()) + 1e-12
+            assert float((p.grad.view(-1).cpu() - want).abs().max()) <= tol
+            assert (p.grad.data_ptr() == snap.data_ptr()) == (dec.regime != orc.PROJECT)
+        seen.add(dec.regime)
+        if take:
+            opt.step()
+    assert orc.PROJECT in seen and orc.SAFE in seen
+    # accumulating into a tensor the controller did not hand out is refused
+    opt.zero_grad(set_to_none=True)
+    torch.nn.functional.mse_loss(net(batches[0]), targets[0]).backward()
+    with pytest.raises(RuntimeError):
+        ctl.step()
+    ctl.close()
