@@ -279,7 +279,17 @@ def time_exchange_mode(wl: Workload, steps: int):
         s_ms = sum(a.elapsed_time(b) for a, b, _ in evs) / len(evs)
         p_ms = sum(b.elapsed_time(c) for _, b, c in evs) / len(evs)
         proj_bpp = 3 * sg if label == "project" else 0
-        out[label] = {"regime": gb.REGIME_NAMES[res.regime], "cos": res.cos, "ms_per_step": s_ms + p_ms,
+        roof = None
+        if proj_bpp:
+            peak, kind = measured_hbm_peak()
+            tr = recorded_traffic("gac_project_kernel_exchange")
+            key = "f32" if sg == 4 else "bf16_dbf16"
+            gbs = wl.params * proj_bpp / (p_ms * 1e-3) / 1e9
+            roof = {"bound": "hbm", "kernel": "gac_project_kernel (exchange)", "achieved": gbs, "peak": peak,
+                    "unit": "GB/s", "frac": gbs / peak, "peak_kind": f"of {kind}",
+                    "algorithmic_bytes_per_launch": wl.params * proj_bpp,
+                    "traffic": (tr[key] * wl.params if tr and key in tr else None)}
+        out[label] = {"roofline": roof,"regime": gb.REGIME_NAMES[res.regime], "cos": res.cos, "ms_per_step": s_ms + p_ms,
                       "stats_ms": s_ms, "project_ms": p_ms, "value": wl.params / ((s_ms + p_ms) * 1e-3),
                       "unit": UNIT, "bytes_per_param": 2 * sg + proj_bpp,
                       "hbm_gbs": wl.params * (2 * sg + proj_bpp) / ((s_ms + p_ms) * 1e-3) / 1e9,
