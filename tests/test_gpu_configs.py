@@ -236,3 +236,68 @@ def test_single_tensor_beyond_32bit_indexing():
         orc.project([g_ref], [d_ref], to_orc_hp(hp), dec, threads=THREADS)
         assert max_ulp(g[lo:hi].cpu(), g_ref) <= 1
         assert torch.equal(d[lo:hi].cpu().view(torch.int16), d_ref.view(torch.int16))
+
+
+# ------------------------------------------------- exchange mode at full size
+
+@pytest.mark.parametrize("workload", ["cfg2_1.5b_f32", "cfg5_14b_f32"])
+def test_config_exchange_mode_two_steps(workload):
+    """Exchange mode on the full-size float32 lists, in the configuration bench.py times: two
+    consecutive projection steps, so that both assignments of the roles run at full size.  The
+    oracle computes the plain rule (d' = g by copy); here g' must appear in the buffers that held
+    d and the buffers that held g must come out untouched, every element."""
+    dims_key, g_dtype, rho, config_id = synth.WORKLOADS[workload]
+    shapes = synth.decoder_tensor_list(synth.DIMS[dims_key])
+    need = synth.list_numel(shapes) * 8 + (12 << 30)
+    free, _ = torch.cuda.mem_get_info()
+    if free < need:
+        pytest.skip(f"needs {need >> 30} GiB of device memory, {free >> 30} GiB free")
+    hp = gb.HParams(state_mode=gb.GAC_STATE_EXCHANGE, **FORCE)
+    ohp = to_orc_hp(gb.HParams(**FORCE))
+    a, b = synth.gradient_list(shapes, rho, config_id, g_dtype, "cuda")       # a: gradient, b: stored direction
+    ctx = gb.gac_init(a, b, hp)
+
+    # step 2: gradient in a, direction in b, g' lands in b
+    dec = orc.decide(oracle_sums_streamed(a, b), ohp)
+    res = gb.gac_stats(ctx, 2)
+    after = gb.gac_project(ctx, coef_override=dec.coef, fetch=True)
+    check_sums(res, dec)
+    check_decision(res, dec)
+    assert dec.regime == orc.PROJECT and (after.g_set, after.out_set) == (gb.GAC_SET_G, gb.GAC_SET_D)
+    for i in range(len(shapes)):
+        (g0,), (d0,) = synth.gradient_list(shapes, rho, config_id, g_dtype, "cuda", indices=[i])
+        assert torch.equal(a[i], g0), f"tensor {i}: the gradient buffers were modified"
+        for lo, hi in slices_of(g0.numel()):
+            g_ref, d_ref = g0[lo:hi].cpu().contiguous(), d0[lo:hi].cpu().contiguous()
+            orc.project([g_ref], [d_ref], ohp, dec, threads=THREADS)
+            u = max_ulp(b[i][lo:hi].cpu(), g_ref)
+            assert u <= 4, f"step 2 tensor {i} [{lo}:{hi}]: g' differs by {u} ulp"
+        del g0, d0
+
+    # step 3: the roles have swapped -- the next gradient goes into b, a is the stored direction
+    assert gb.gac_next_gradient_set(ctx) == gb.GAC_SET_D
+    sigma = synth.per_tensor_scales(config_id, len(shapes))
+    gen = torch.Generator(device="cuda").manual_seed(4242)
+    scratch = torch.empty(max(n for _, n in shapes), dtype=torch.float32, device="cuda")
+    synth.refresh_gradient_list(b, a, sigma, rho, gen, scratch)
+    del scratch
+    dec = orc.decide(oracle_sums_streamed(b, a), ohp)
+    res = gb.gac_stats(ctx, 3)
+    after = gb.gac_project(ctx, coef_override=dec.coef, fetch=True)
+    check_sums(res, dec)
+    check_decision(res, dec)
+    assert dec.regime == orc.PROJECT and (after.g_set, after.out_set) == (gb.GAC_SET_D, gb.GAC_SET_G)
+    assert abs(res.cos - rho) < 2e-3
+    for i in range(len(shapes)):
+        (d0,), _ = synth.gradient_list(shapes, rho, config_id, g_dtype, "cuda", indices=[i])   # a before this step
+        for lo, hi in slices_of(d0.numel()):
+            g_ref, d_ref = b[i][lo:hi].cpu().contiguous(), d0[lo:hi].cpu().contiguous()
+            g_in = g_ref.clone()
+            orc.project([g_ref], [d_ref], ohp, dec, threads=THREADS)
+            u = max_ulp(a[i][lo:hi].cpu(), g_ref)
+            assert u <= 4, f"step 3 tensor {i} [{lo}:{hi}]: g' differs by {u} ulp"
+            assert torch.equal(d_ref, g_in)        # the rule's new direction is the raw gradient: b, untouched
+        del d0
+    gb.gac_free(ctx)
+    del a, b
+    torch.cuda.empty_cache()
