@@ -299,11 +299,14 @@ def time_exchange_mode(wl: Workload, steps: int):
     return out
 
 
-def time_fused_adamw(wl: Workload, steps: int):
+def time_fused_adamw(wl: Workload, steps: int, exchange: bool = False):
     """stats + the projection fused with AdamW (Table 2 values): the update goes
-    straight into p, m, v and g' is never written.  Moves (sg+4) + (sg+4+12) read
-    + 16 written bytes per parameter."""
+    straight into p, m, v and g' is never written.  Moves (sg+sd) + (sg+sd+12) read
+    + (sd+12) written bytes per parameter; in exchange mode the stored direction
+    is not written either (12 written)."""
     gb = wl.gb
+    if exchange and wl.g_dtype != wl.d_dtype:
+        return {"skipped": "exchange mode needs g and d of one element type"}
     free, _ = torch.cuda.mem_get_info()
     need = wl.params * 12 + (2 << 30)
     if free < need:
@@ -311,12 +314,17 @@ def time_fused_adamw(wl: Workload, steps: int):
     p = [torch.randn(t.numel(), device=wl.device) * 0.02 for t in wl.g]
     m = [torch.zeros(t.numel(), device=wl.device) for t in wl.g]
     v = [torch.zeros(t.numel(), device=wl.device) for t in wl.g]
-    ctx = gb.gac_init(wl.g, wl.d, gb.HParams(**FORCE))
+    sets = [wl.g, wl.d]
+    mode = gb.GAC_STATE_EXCHANGE if exchange else gb.GAC_STATE_RAW
+    ctx = gb.gac_init(wl.g, wl.d, gb.HParams(state_mode=mode, **FORCE))
     gb.gac_attach_adamw(ctx, p, m, v, 0)
     opt = gb.AdamW()
     step_no, evs = 1, []
-    for i in range(3 + steps):
-        wl.refresh()
+    for i in range(3 + steps + 1):
+        gi = gb.gac_next_gradient_set(ctx)          # always the g buffers outside exchange mode
+        synth.refresh_gradient_list(sets[gi], sets[gi ^ 1], wl.sigma, wl.rho, wl.gen, wl.scratch)
+        if i == 3 + steps:
+            break
         step_no += 1
         e = [torch.cuda.Event(enable_timing=True) for _ in range(3)]
         e[0].record()
@@ -329,16 +337,21 @@ def time_fused_adamw(wl: Workload, steps: int):
     torch.cuda.synchronize()
     gb.gac_stats(ctx, step_no + 1, fetch=False)
     res = gb.gac_project_adamw(ctx, opt, fetch=True)
+    # leave the workload usable by the legs that follow: wl.g a gradient against wl.d
+    synth.refresh_gradient_list(wl.g, wl.d, wl.sigma, wl.rho, wl.gen, wl.scratch)
+    torch.cuda.synchronize()
     gb.gac_free(ctx)
     s_ms = sum(a.elapsed_time(b) for a, b, _ in evs) / len(evs)
     f_ms = sum(b.elapsed_time(c) for _, b, c in evs) / len(evs)
     sg = 2 if wl.g_dtype == torch.bfloat16 else 4
-    fused_bytes = wl.params * ((sg + 4 + 12) + 16)
+    sd = 2 if wl.d_dtype == torch.bfloat16 else 4
+    bpp = (sg + sd + 12) + (12 if exchange else sd + 12)
+    fused_bytes = wl.params * bpp
     del p, m, v
     torch.cuda.empty_cache()
     return {"ms_per_step": s_ms + f_ms, "stats_ms": s_ms, "fused_ms": f_ms,
             "value": wl.params / ((s_ms + f_ms) * 1e-3), "unit": UNIT,
-            "fused_bytes_per_param": (sg + 4 + 12) + 16,
+            "fused_bytes_per_param": bpp,
             "fused_kernel_gbs": fused_bytes / (f_ms * 1e-3) / 1e9,
             "applied_steps": res.applied_steps, "regime": gb.REGIME_NAMES[res.regime]}
 
@@ -608,6 +621,8 @@ def main():
         line["unchanged_regime"] = time_unchanged_regime(wl, min(args.steps, 10))
     if world == 1 and args.adamw:
         line["fused_adamw"] = time_fused_adamw(wl, min(args.steps, 10))
+        if wl.g_dtype == wl.d_dtype:
+            line["fused_adamw_exchange"] = time_fused_adamw(wl, min(args.steps, 10), exchange=True)
     if world == 1 and wl.g_dtype == wl.d_dtype:
         line["exchange_mode"] = time_exchange_mode(wl, min(args.steps, 10))
     if not args.no_e2e:

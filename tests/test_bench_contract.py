@@ -44,6 +44,22 @@ def test_library_arm_line_on_a_small_list():
     assert {"sm_mhz", "sm_max_mhz", "reasons"} <= set(d["clocks"])
     assert d["also"]["regime_check"]["regime"] == "project"
     assert d["unchanged_regime"]["regime"] == "violation"
+    # the float32 list also reports exchange mode: fewer bytes per parameter, same regimes
+    x = d["also"]["exchange_mode"]
+    assert x["project"]["regime"] == "project" and x["project"]["bytes_per_param"] == 20
+    assert x["unchanged"]["regime"] == "violation" and x["unchanged"]["bytes_per_param"] == 8
+    assert x["project"]["roofline"]["bound"] == "hbm"
+
+
+@pytest.mark.gpu
+def test_fused_adamw_legs_on_a_small_list():
+    d = run_bench("--workload", "small_f32", "--also", "none", "--steps", "3", "--warmup", "3", "--adamw",
+                  "--no-e2e", "--no-cpu-baseline")
+    assert d["fused_adamw"]["regime"] == "project" and d["fused_adamw"]["fused_bytes_per_param"] == 36
+    assert d["fused_adamw_exchange"]["regime"] == "project"
+    assert d["fused_adamw_exchange"]["fused_bytes_per_param"] == 32
+    assert d["fused_adamw"]["applied_steps"] == d["fused_adamw_exchange"]["applied_steps"] > 0
+    assert d["exchange_mode"]["project"]["regime"] == "project"
 
 
 @pytest.mark.gpu
