@@ -481,8 +481,8 @@ def run_reference(args):
     name = args.workload
     # calibrate so that warmup+steps passes end within about two minutes
     probe = time_oracle(name, 8_000_000, 1, 0)
-    budget_s = 100.0 / max(1, args.steps + args.warmup)
-    target = int(min(2_000_000_000, max(8_000_000, probe["value"] * budget_s)))
+    pass_seconds = 100.0 / max(1, args.steps + args.warmup)
+    target = int(min(2_000_000_000, max(8_000_000, probe["value"] * pass_seconds)))
     cb = time_oracle(name, target, args.steps, args.warmup)
     dims_key, g_dtype, rho, config_id = synth.WORKLOADS[name]
     line = {"impl": "reference", "metric": METRIC, "value": cb["value"], "unit": UNIT,
