@@ -135,7 +135,8 @@ void gac_default_hparams(gac_hparams *hp);
  *   n            number of tensors, >= 1; every numel >= 1
  *   g_dtype/d_dtype  supported pairs: (F32,F32), (BF16,F32), and (BF16,BF16) -- a
  *                snapshot of half the size (App. A.2 "Memory footprint"), still an
- *                exact copy of the bfloat16 gradient
+ *                exact copy of the bfloat16 gradient.  state_mode EXCHANGE needs
+ *                g_dtype == d_dtype (GAC_ERR_DTYPE otherwise)
  *   hp           host pointer; copied
  *   cuda_device  ordinal of the device that owns g and d
  * Allocates device and pinned memory (not capturable in a CUDA graph).
@@ -188,7 +189,8 @@ int gac_decide(gac_ctx *ctx, void *cuda_stream, const double *sums_in, gac_resul
  *   SAFE             g untouched (Algorithm 1: ordinary update)
  *   VIOLATION        g untouched, or zeroed if zero_on_violation; the caller
  *                    skips its optimizer step (Algorithm 1: theta_t = theta_{t-1})
- *   every regime     d'_i = g_i, the raw gradient (state_mode RAW)
+ *   every regime     d'_i = g_i, the raw gradient (state_mode RAW; EXCHANGE reaches the
+ *                    same state without this copy, see "Exchange mode" below)
  *   nonfinite        neither g nor d is written
  * Must follow a gac_stats / gac_decide of the same step (else STATE).
  *   coef_override    host pointer to one float, or NULL.  When given, it
