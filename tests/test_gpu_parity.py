@@ -472,3 +472,31 @@ def test_rebind_to_moved_buffers_keeps_the_step_sequence():
     with pytest.raises(gb.GacError):
         gb.gac_rebind(ctx, g2[:-1], d2[:-1])
     gb.gac_free(ctx)
+
+
+@pytest.mark.parametrize("g_dtype", [torch.float32, torch.bfloat16], ids=["f32", "bf16"])
+def test_power_of_two_rescaling_on_device(g_dtype):
+    """App. A.1: the cosine does not depend on the gradient's scale.  With eps = 0, rescaling g and d
+    by powers of two (exact in binary floating point, far from over- and underflow of the sums in
+    binary64) must leave cosine, regime and alpha bit-identical on the device, and scale g' exactly."""
+    n = 40_001
+    g, d = rand_pair(n, 0.6, seed=21, g_dtype=g_dtype, scale=1.0)
+    hp = gb.HParams(c_low=0.05, c_high=2.0, eps=0.0)
+    base = None
+    # the multiplier of d is one binary32 number that scales as 2^(eg - ed): kept within binary32's range
+    for eg, ed in [(0, 0), (-90, 0), (60, 0), (0, -100), (0, 90), (-80, -70), (50, 50)]:
+        gs = (g.double() * 2.0 ** eg).to(g_dtype)
+        ds = (d.double() * 2.0 ** ed).float()
+        assert torch.isfinite(gs.float()).all() and (gs.float().abs() >= 2.0 ** -120)[g.float() != 0].all()
+        res, dec, gg, dg, gr, dr = step_both([gs], [ds], hp, same_coef=False)
+        check_sums(res, dec, rel=1e-13)
+        check_decision(res, dec)
+        assert (res.cos, res.regime, res.alpha) == (dec.cos, dec.regime, dec.alpha)
+        out = (gg[0].cpu().double() * 2.0 ** -eg)
+        if base is None:
+            base = (res.cos, res.regime, res.alpha, out)
+        else:
+            assert (res.cos, res.regime, res.alpha) == base[:3]
+            # g' = g + k d with k = (alpha - 1) dot/dd scaling as 2^(eg - ed): every term scales by 2^eg
+            assert torch.equal(out, base[3]), (eg, ed)
+        assert torch.equal(dg[0].cpu(), gs.float())
