@@ -219,7 +219,8 @@ int gac_project(gac_ctx *ctx, void *cuda_stream, const float *coef_override, gac
  * unconditional, so the caller can follow it without reading anything back:
  * step by step the gradient alternates between the two sets, starting with the
  * `g` pointers given to gac_init (gac_rebind starts over with the new `g`).
- * gac_next_gradient_set reports it.  The record says where the outgoing gradient
+ * gac_next_gradient_set reports it (which set is g is a launch argument: a step
+ * captured in a CUDA graph serves every second step).  The record says where the outgoing gradient
  * is (`out_set`).  A non-finite step writes nothing; since the roles swap all the
  * same, the stored direction is lost with it and the following step is taken
  * against the zero reference (`ref_lost`), as the first step is.

@@ -339,3 +339,50 @@ def test_exchange_mode_random_list_structures(seed):
         for b, o, n in zip(bufs[k], offs, sizes):
             assert bool((b[:o[k]] == 3.0).all()) and bool((b[o[k] + n:] == 3.0).all())
     gb.gac_free(ctx)
+
+
+def test_exchange_mode_steps_replayed_from_cuda_graphs():
+    """The role of each buffer set is a launch argument, so one captured step serves every second
+    step: two graphs (gradient in the `g` set, gradient in the `d` set) replayed in turn give what
+    direct calls give."""
+    n = 1 << 20
+    hp = gb.HParams(state_mode=gb.GAC_STATE_EXCHANGE, c_low=0.05, c_high=2.0)
+    ohp = raw_hp(hp)
+    g0, d0 = synth.flat_pair_with_cosine(n, 0.9, s=1.0, seed=0)
+    sets = [[g0.cuda()], [d0.cuda()]]
+    ctx = gb.gac_init(sets[0], sets[1], hp)
+    gb.gac_stats(ctx, 2, fetch=False)            # two warm-up steps outside capture: roles back where they began
+    gb.gac_project(ctx)
+    gb.gac_stats(ctx, 3, fetch=False)
+    gb.gac_project(ctx)
+    torch.cuda.synchronize()
+    graphs = []
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        for k in range(2):
+            assert gb.gac_next_gradient_set(ctx) == k
+            gr = torch.cuda.CUDAGraph()
+            gr.capture_begin()
+            gb.gac_stats(ctx, 4 + k, fetch=False)
+            gb.gac_project(ctx)
+            gr.capture_end()
+            graphs.append(gr)
+    torch.cuda.current_stream().wait_stream(side)
+    d_ref = [d0.clone()]
+    sets[1][0].copy_(d0)
+    for t in range(4):
+        gi = t % 2
+        gen = torch.Generator().manual_seed(50 + t)
+        g_new = (0.6 * d_ref[0] + 0.8 * d_ref[0].std() * torch.randn(n, generator=gen))
+        sets[gi][0].copy_(g_new)
+        graphs[gi].replay()
+        torch.cuda.synchronize()
+        g_ref = [g_new.clone()]
+        dec = orc.step(g_ref, d_ref, ohp)               # d_ref <- raw gradient
+        assert dec.regime == orc.PROJECT
+        assert same_bits(sets[gi][0], g_new)            # untouched: it is the stored direction now
+        out = sets[gi ^ 1][0].cpu()
+        # the coefficient is the library's own here (nothing can be overridden inside a replay)
+        assert float((out.double() - g_ref[0].double()).abs().max()) <= 2e-7 * float(g_new.abs().max())
+    gb.gac_free(ctx)
