@@ -13,6 +13,10 @@ step, summed over the K timed steps; between steps a FRESH gradient with the
 configured cosine to the stored direction is written into g (as the backward
 pass of a training loop would), outside the timed events; that write also
 evicts the 126 MB L2.  Prints one JSON line.
+
+--gpus N > 1 without a launcher's environment starts N ranks by itself (one
+process per GPU, NCCL, a free port on 127.0.0.1); under an external launcher
+(RANK / WORLD_SIZE / LOCAL_RANK set) it is one of those ranks.
 """
 from __future__ import annotations
 
@@ -22,7 +26,9 @@ import hashlib
 import json
 import math
 import os
+import socket
 import statistics
+import subprocess
 import sys
 import threading
 import time
@@ -138,12 +144,55 @@ def recorded_traffic(kernel: str):
         return None
 
 
+# ------------------------------------------------------------------ launcher
+
+def free_port() -> int:
+    with socket.socket() as sock:
+        sock.bind(("127.0.0.1", 0))
+        return sock.getsockname()[1]
+
+
+def rank_environment(n: int, rank: int, port: int, base=None) -> dict:
+    """Environment of rank `rank` of an n-rank single-node job, as torch.distributed's
+    env:// rendezvous reads it.  Everything else is inherited (NCCL settings included)."""
+    env = dict(os.environ if base is None else base)
+    env.update({"RANK": str(rank), "LOCAL_RANK": str(rank), "WORLD_SIZE": str(n),
+                "LOCAL_WORLD_SIZE": str(n), "MASTER_ADDR": "127.0.0.1", "MASTER_PORT": str(port)})
+    return env
+
+
+def spawn_ranks(n: int, argv, worker=None, stdout=None) -> int:
+    """Starts n copies of this script (or of `worker`, a command prefix), one per GPU, and waits.
+    Rank 0 prints the JSON line on the inherited stdout.  If a rank fails the others are
+    terminated and its exit code is returned."""
+    worker = worker or [sys.executable, os.path.abspath(__file__)]
+    port = free_port()
+    procs = [subprocess.Popen(list(worker) + list(argv), env=rank_environment(n, r, port), stdout=stdout)
+             for r in range(n)]
+    rc = 0
+    pending = set(range(n))
+    while pending:
+        for r in sorted(pending):
+            code = procs[r].poll()
+            if code is None:
+                continue
+            pending.discard(r)
+            if code != 0 and rc == 0:
+                rc = code
+                for q in pending:
+                    procs[q].terminate()
+        time.sleep(0.05)
+    return rc
+
+
 # --------------------------------------------------------------- GPU workload
 
 class Workload:
-    def __init__(self, name: str, device, world: int, clip: float = 0.0, sharded: bool = False):
+    def __init__(self, name: str, device, world: int, clip: float = 0.0, sharded: bool = False,
+                 peer_exchange: bool = False):
         from paper_2603_01501_b200 import binding as gb
-        self.gb = gb
+        from paper_2603_01501_b200 import sharding
+        self.gb, self.sharding = gb, sharding
         dims_key, self.g_dtype, self.rho, self.config_id = synth.WORKLOADS[name]
         self.name, self.device, self.world = name, device, world
         self.shapes = synth.decoder_tensor_list(synth.DIMS[dims_key])
@@ -160,6 +209,9 @@ class Workload:
         self.step_no = 1      # the stored direction already holds g_{t-1}
         self.sharded = sharded or world > 1     # local sums -> all-reduce -> decision (App. A.1)
         self.sums = torch.zeros(3, dtype=torch.float64, device=device) if self.sharded else None
+        self.peer_exchange = bool(peer_exchange and self.sharded)
+        if self.peer_exchange:      # the kernels exchange the three sums themselves instead of NCCL
+            self.sharding.attach_peer_exchange(gb, self.ctx)
 
     def refresh(self):
         synth.refresh_gradient_list(self.g, self.d, self.sigma, self.rho, self.gen, self.scratch)
@@ -172,14 +224,13 @@ class Workload:
             ev[0].record()
         if self.sharded:
             # sharded form (App. A.1): local sums, ONE all-reduce of three numbers, same decision on every rank
-            gb.gac_stats_partial(self.ctx, self.step_no, self.sums)
-            torch.distributed.all_reduce(self.sums)
-            gb.gac_decide(self.ctx, self.sums, fetch=False)
+            self.sharding.sharded_step(gb, self.ctx, self.step_no, self.sums,
+                                       mark=(ev[1].record if ev else None), peer_exchange=self.peer_exchange)
         else:
             gb.gac_stats(self.ctx, self.step_no, fetch=False)
-        if ev:
-            ev[1].record()
-        gb.gac_project(self.ctx)
+            if ev:
+                ev[1].record()
+            gb.gac_project(self.ctx)
         if ev:
             ev[2].record()
 
@@ -299,7 +350,7 @@ def time_exchange_mode(wl: Workload, steps: int):
     return out
 
 
-def time_fused_adamw(wl: Workload, steps: int, exchange: bool = False):
+def time_fused_adamw(wl: Workload, steps: int, exchange: bool = False, peak=None, peak_kind="measured"):
     """stats + the projection fused with AdamW (Table 2 values): the update goes
     straight into p, m, v and g' is never written.  Moves (sg+sd) + (sg+sd+12) read
     + (sd+12) written bytes per parameter; in exchange mode the stored direction
@@ -349,10 +400,19 @@ def time_fused_adamw(wl: Workload, steps: int, exchange: bool = False):
     fused_bytes = wl.params * bpp
     del p, m, v
     torch.cuda.empty_cache()
-    return {"ms_per_step": s_ms + f_ms, "stats_ms": s_ms, "fused_ms": f_ms,
+    gbs = fused_bytes / (f_ms * 1e-3) / 1e9
+    if peak is None:
+        peak, peak_kind = measured_hbm_peak()
+    tr = recorded_traffic("gac_adamw_kernel_exchange" if exchange else "gac_adamw_kernel")
+    key = dtype_name(wl.g_dtype) + ("_dbf16" if wl.d_dtype != torch.float32 else "")
+    return {"ms_per_step": s_ms + f_ms, "stats_ms": s_ms, "fused_ms": f_ms, "steps": len(evs),
             "value": wl.params / ((s_ms + f_ms) * 1e-3), "unit": UNIT,
             "fused_bytes_per_param": bpp,
-            "fused_kernel_gbs": fused_bytes / (f_ms * 1e-3) / 1e9,
+            "fused_kernel_gbs": gbs,
+            "roofline": {"bound": "hbm", "kernel": "gac_adamw_kernel" + (" (exchange)" if exchange else ""),
+                         "achieved": gbs, "peak": peak, "unit": "GB/s", "frac": gbs / peak,
+                         "peak_kind": f"of {peak_kind}", "algorithmic_bytes_per_launch": fused_bytes,
+                         "traffic": (tr[key] * wl.params if tr and key in tr else None)},
             "applied_steps": res.applied_steps, "regime": gb.REGIME_NAMES[res.regime]}
 
 
@@ -371,12 +431,10 @@ def check_regime(wl: Workload):
     gb = wl.gb
     wl.step_no += 1
     if wl.sharded:
-        gb.gac_stats_partial(wl.ctx, wl.step_no, wl.sums)
-        torch.distributed.all_reduce(wl.sums)
-        res = gb.gac_decide(wl.ctx, wl.sums)
+        res = wl.sharding.sharded_step(gb, wl.ctx, wl.step_no, wl.sums, fetch=True, peer_exchange=wl.peer_exchange)
     else:
         res = gb.gac_stats(wl.ctx, wl.step_no)
-    gb.gac_project(wl.ctx)
+        gb.gac_project(wl.ctx)
     torch.cuda.synchronize()
     return res
 
@@ -432,15 +490,27 @@ def time_e2e(wl: Workload, steps: int, warmup: int):
 
 # ------------------------------------------------------------- CPU baseline
 
+# Both arms time the oracle on the SAME bounded samples of the workload, so their figures agree:
+# all host cores on the first ALL_CORE_SAMPLE parameters after the embedding (the per-layer mix of
+# small and large tensors), one thread on the first ONE_THREAD_SAMPLE of those.
+ALL_CORE_SAMPLE = 1_000_000_000
+ONE_THREAD_SAMPLE = 64_000_000
+
+
+def host_cores() -> int:
+    return len(os.sched_getaffinity(0)) if hasattr(os, "sched_getaffinity") else (os.cpu_count() or 1)
+
+
 def oracle_sample(name: str, target_elems: int):
     """A prefix of the workload's tensor list (whole tensors, the last one cut),
     generated on the CPU with the list's recipe."""
     dims_key, g_dtype, rho, config_id = synth.WORKLOADS[name]
     shapes = synth.decoder_tensor_list(synth.DIMS[dims_key])
-    # skip the embedding so that the sample holds the per-layer mix of small and large tensors
     sig = synth.per_tensor_scales(config_id, len(shapes))
+    # skip the embedding so that the sample holds the per-layer mix of small and large tensors
+    first = 1 if len(shapes) > 1 else 0
     gs, ds, total, used = [], [], 0, 0
-    for i in range(1, len(shapes)):
+    for i in range(first, len(shapes)):
         n = min(shapes[i][1], target_elems - total)
         if n <= 0:
             break
@@ -452,10 +522,10 @@ def oracle_sample(name: str, target_elems: int):
     return gs, ds, total, used
 
 
-def time_oracle(name: str, target_elems: int, steps: int, warmup: int):
+def time_oracle_on(sample, name: str, threads: int, steps: int, warmup: int):
+    """Wall clock of the oracle's whole step (stats, decision, projection, state refresh) on a sample."""
     from oracle import gac_oracle as orc
-    threads = len(os.sched_getaffinity(0)) if hasattr(os, "sched_getaffinity") else os.cpu_count()
-    gs, ds, total, used = oracle_sample(name, target_elems)
+    gs, ds, total, used = sample
     hp = orc.HParams(**FORCE)
     times = []
     for i in range(warmup + steps):
@@ -468,42 +538,71 @@ def time_oracle(name: str, target_elems: int, steps: int, warmup: int):
             times.append(dt)
     sec = sum(times) / len(times)
     return {"value": total / sec, "unit": UNIT, "cores": threads, "kind": "oracle",
-            "sample": f"tensors 1..{used} of the {name} list ({total} params), stats+project, "
-                      f"{steps} timed passes of {sec:.2f} s", "seconds_per_pass": sec}
+            "sample": f"first {used} tensors after the embedding of the {name} list ({total} params, the last "
+                      f"tensor cut), stats+project, {steps} timed passes of {sec:.2f} s",
+            "seconds_per_pass": sec}
+
+
+def sample_sizes(name: str):
+    dims_key = synth.WORKLOADS[name][0]
+    shapes = synth.decoder_tensor_list(synth.DIMS[dims_key])
+    avail = synth.list_numel(shapes[1:] if len(shapes) > 1 else shapes)
+    return min(ALL_CORE_SAMPLE, avail), min(ONE_THREAD_SAMPLE, avail)
+
+
+def cpu_baseline(name: str, passes: int = 3):
+    """The oracle as it stands on this host: all cores, and one thread on a prefix of the same sample."""
+    n_all, n_one = sample_sizes(name)
+    sample = oracle_sample(name, n_all)
+    cores = host_cores()
+    allc = time_oracle_on(sample, name, cores, passes, 1)
+    one = time_oracle_on(oracle_sample(name, n_one), name, 1, passes, 1)
+    out = {k: allc[k] for k in ("value", "unit", "cores", "kind", "sample")}
+    out["single_thread"] = {k: one[k] for k in ("value", "unit", "cores", "sample")}
+    return out
 
 
 def run_reference(args):
     """The CPU oracle as it stands, on the host cores, on the same workload
-    definition (a bounded sample of it per step)."""
+    definition: every step is one pass over the bounded sample that the library
+    arm's `cpu_baseline` uses (shrunk only if K + W passes would not end within
+    a few minutes)."""
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return 0
     name = args.workload
-    # calibrate so that warmup+steps passes end within about two minutes
-    probe = time_oracle(name, 8_000_000, 1, 0)
-    pass_seconds = 100.0 / max(1, args.steps + args.warmup)
-    target = int(min(2_000_000_000, max(8_000_000, probe["value"] * pass_seconds)))
-    cb = time_oracle(name, target, args.steps, args.warmup)
-    dims_key, g_dtype, rho, config_id = synth.WORKLOADS[name]
+    cores = host_cores()
+    n_all, n_one = sample_sizes(name)
+    probe = time_oracle_on(oracle_sample(name, min(n_all, 8_000_000)), name, cores, 1, 0)
+    budget_s = 150.0 / max(1, args.steps + args.warmup)
+    target = int(min(n_all, max(8_000_000, probe["value"] * budget_s)))
+    cb = time_oracle_on(oracle_sample(name, target), name, cores, args.steps, args.warmup)
+    one = time_oracle_on(oracle_sample(name, n_one), name, 1, 2, 1)
+    config = workload_config(name)
+    config["timing"] = "host wall clock (time.perf_counter) around each oracle pass; no GPU is used"
+    base = {k: cb[k] for k in ("value", "unit", "cores", "kind", "sample")}
+    base["single_thread"] = {k: one[k] for k in ("value", "unit", "cores", "sample")}
     line = {"impl": "reference", "metric": METRIC, "value": cb["value"], "unit": UNIT,
             "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup,
             "ms_per_step": cb["seconds_per_pass"] * 1e3, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-            "config": workload_config(name, None),
-            "cpu_baseline": {k: cb[k] for k in ("value", "unit", "cores", "kind", "sample")},
+            "config": config, "cpu_baseline": base,
             "e2e": {"value": cb["value"], "unit": UNIT, "h2d_bytes_per_step": 0,
                     "d2h_bytes_per_step": 0}}
     print(json.dumps(line))
     return 0
 
 
-def workload_config(name: str, wl):
+def dtype_name(t) -> str:
+    return "bf16" if t == torch.bfloat16 else "f32"
+
+
+def workload_config(name: str):
     dims_key, g_dtype, rho, config_id = synth.WORKLOADS[name]
     shapes = synth.decoder_tensor_list(synth.DIMS[dims_key])
     d_dtype = synth.WORKLOAD_D_DTYPE.get(name, torch.float32)
     return {"workload": f"{name}: {dims_key} decoder-shaped gradient list, "
-                        f"{'bf16' if g_dtype == torch.bfloat16 else 'f32'} g / "
-                        f"{'bf16' if d_dtype == torch.bfloat16 else 'f32'} d, target cosine {rho}, "
+                        f"{dtype_name(g_dtype)} g / {dtype_name(d_dtype)} d, target cosine {rho}, "
                         f"projection regime forced with c_low=0.05 c_high=2.0",
             "params_per_gpu": synth.list_numel(shapes), "tensors": len(shapes),
             "bytes_per_param": 3 * bytes_per_param(g_dtype, d_dtype),
@@ -543,6 +642,64 @@ def summarize(wl: Workload, s_ms, p_ms, peak, peak_kind):
     }
 
 
+def time_graph_replay(wl: Workload, replays: int = 200):
+    """One step (both launches, no host read-back) captured in a CUDA graph and replayed:
+    what a launch-bound list costs once the launch overhead of two direct calls is gone."""
+    gb = wl.gb
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        wl.step()
+        side.synchronize()
+        graph = torch.cuda.CUDAGraph()
+        graph.capture_begin()
+        wl.step()
+        graph.capture_end()
+        for _ in range(5):
+            graph.replay()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        for _ in range(replays):
+            graph.replay()
+        b.record()
+        side.synchronize()
+    torch.cuda.current_stream().wait_stream(side)
+    return a.elapsed_time(b) / replays * 1e3     # microseconds per step
+
+
+def time_other(name: str, device, steps: int, peak: float, adamw: bool = False):
+    """A further workload, timed the same way (fewer steps): a compact record."""
+    gb_need = synth.list_numel(synth.decoder_tensor_list(synth.DIMS[synth.WORKLOADS[name][0]])) * \
+        bytes_per_param(synth.WORKLOADS[name][1], synth.WORKLOAD_D_DTYPE.get(name, torch.float32)) + (6 << 30)
+    free, _ = torch.cuda.mem_get_info()
+    if free < gb_need:
+        return {"skipped": f"needs {gb_need} bytes of device memory, {free} free"}
+    wl = Workload(name, device, 1)
+    s_ms, p_ms = time_steps(wl, steps, 3)
+    res = check_regime(wl)
+    bpp = bytes_per_param(wl.g_dtype, wl.d_dtype)
+    s_avg, p_avg = sum(s_ms) / len(s_ms), sum(p_ms) / len(p_ms)
+    ms = s_avg + p_avg
+    out = {"params": wl.params, "steps": steps, "ms_per_step": ms, "stats_ms": s_avg, "project_ms": p_avg,
+           "value": wl.params / (ms * 1e-3), "unit": UNIT, "bytes_per_param": 3 * bpp,
+           "hbm_gbs": 3 * bpp * wl.params / (ms * 1e-3) / 1e9,
+           "stats_gbs": bpp * wl.params / (s_avg * 1e-3) / 1e9,
+           "project_gbs": 2 * bpp * wl.params / (p_avg * 1e-3) / 1e9,
+           "stats_frac_of_measured_copy": bpp * wl.params / (s_avg * 1e-3) / 1e9 / peak,
+           "project_frac_of_measured_copy": 2 * bpp * wl.params / (p_avg * 1e-3) / 1e9 / peak,
+           "regime_check": {"cos": res.cos, "regime": wl.gb.REGIME_NAMES[res.regime]}}
+    if 3 * bpp * wl.params < (126 << 20):
+        out["note"] = ("launch-bound: the whole step moves less than the 126 MB L2 holds, so this is not a "
+                       "roofline point")
+        out["graph_replay_us_per_step"] = time_graph_replay(wl)
+    if adamw:
+        out["fused_adamw"] = time_fused_adamw(wl, steps, peak=peak)
+        if wl.g_dtype == wl.d_dtype:
+            out["fused_adamw_exchange"] = time_fused_adamw(wl, steps, exchange=True, peak=peak)
+    wl.close()
+    return out
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -552,24 +709,38 @@ def main():
     ap.add_argument("--workload", default="cfg3_7b_bf16", choices=sorted(synth.WORKLOADS))
     ap.add_argument("--also", default="cfg5_14b_f32",
                     help="second workload reported under 'also' (1 GPU only); 'none' to skip")
+    ap.add_argument("--others", default="cfg1_flat_f32,cfg2_1.5b_f32,cfg3_7b_bf16_dbf16",
+                    help="further workloads reported compactly under 'others' (1 GPU only); 'none' to skip")
     ap.add_argument("--clip", type=float, default=0.0,
                     help="fold global-norm clipping with this max norm into the projection pass (0 = off)")
     ap.add_argument("--sharded", action="store_true",
                     help="use the sharded call sequence (local sums, NCCL all-reduce of 3 doubles, decision) "
                          "even on one GPU; always on for --gpus > 1")
-    ap.add_argument("--adamw", action="store_true",
-                    help="also time the projection fused with AdamW on the main workload (1 GPU)")
+    ap.add_argument("--exchange", default="nccl", choices=["nccl", "peer"],
+                    help="how the sharded form sums its three numbers across ranks: NCCL's all-reduce (default) or "
+                         "the library's own peer stores in the reduction's epilogue (needs symmetric memory)")
+    ap.add_argument("--no-adamw", action="store_true",
+                    help="skip the legs that time the projection fused with AdamW (1 GPU)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
     if args.warmup < 3:
         args.warmup = 3
+    if args.gpus < 1:
+        raise SystemExit("--gpus must be >= 1")
 
     if args.impl == "reference":
         return run_reference(args)
 
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device: the GAC path has no CPU fallback")
+    if "WORLD_SIZE" not in os.environ and args.gpus > 1:
+        # no launcher around us: become the launcher of one rank per GPU
+        have = torch.cuda.device_count()
+        if args.gpus > have:
+            raise SystemExit(f"--gpus {args.gpus}: only {have} CUDA device(s) are visible")
+        return spawn_ranks(args.gpus, sys.argv[1:])
+
     from paper_2603_01501_b200 import binding as gb
     gb.load_library()
 
@@ -580,11 +751,14 @@ def main():
     device = torch.device("cuda", local_rank)
     if world > 1 or args.sharded:
         os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
-        os.environ.setdefault("MASTER_PORT", "29577")
+        if "MASTER_PORT" not in os.environ:
+            if world > 1:
+                raise SystemExit("WORLD_SIZE > 1 needs MASTER_PORT from the launcher")
+            os.environ["MASTER_PORT"] = str(free_port())
         torch.distributed.init_process_group("nccl", device_id=device, rank=rank, world_size=world)
     peak, peak_kind = measured_hbm_peak()
 
-    wl = Workload(args.workload, device, world, args.clip, args.sharded)
+    wl = Workload(args.workload, device, world, args.clip, args.sharded, args.exchange == "peer")
     sampler = ClockSampler(nvml_index(local_rank))
     wall0 = time.perf_counter()
     s_ms, p_ms = time_steps(wl, args.steps, args.warmup, sampler)
@@ -600,8 +774,9 @@ def main():
     info = gb.gac_get_info(wl.ctx)
     line = {"metric": METRIC, "value": wl.params * world / (ms_per_step * 1e-3), "unit": UNIT,
             "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_per_step,
-            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32",
-            "data": "synthetic", "config": workload_config(args.workload, wl),
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": f"{dtype_name(wl.g_dtype)} g / {dtype_name(wl.d_dtype)} d, f64 sums, f32 fma",
+            "data": "synthetic", "config": workload_config(args.workload),
             "hbm_gbs": summ["hbm_gbs"] , "frac_of_nominal_8TBs": summ["hbm_gbs"] / NOMINAL_HBM_GBS,
             "stats_ms": summ["stats_ms"], "project_ms": summ["project_ms"],
             "best_ms_per_step": summ["best_ms_per_step"],
@@ -613,18 +788,22 @@ def main():
             "gpu_launches": (3 if wl.sharded else 2) * args.steps,
             "clocks": sampler.summary(), "roofline": summ["roofline"],
             "roofline_stats": summ["roofline_stats"], "wall_s_timed_loop": wall}
+    how = ("the three sums exchanged by peer stores in the reduction's epilogue" if wl.peer_exchange
+           else "one NCCL all-reduce of 3 doubles per step")
     if world > 1:
-        line["config"]["parallelism"] = (f"dp{world}: every rank holds one list as its gradient shard; "
-                                         "one NCCL all-reduce of 3 doubles per step")
+        line["config"]["parallelism"] = f"dp{world}: every rank holds one list as its gradient shard; {how}"
+    elif wl.sharded:
+        line["config"]["parallelism"] = f"dp1: the sharded call sequence in a one-rank group; {how}"
 
+    few = min(args.steps, 10)
     if world == 1:
-        line["unchanged_regime"] = time_unchanged_regime(wl, min(args.steps, 10))
-    if world == 1 and args.adamw:
-        line["fused_adamw"] = time_fused_adamw(wl, min(args.steps, 10))
+        line["unchanged_regime"] = time_unchanged_regime(wl, few)
+    if world == 1 and not args.no_adamw:
+        line["fused_adamw"] = time_fused_adamw(wl, few, peak=peak, peak_kind=peak_kind)
         if wl.g_dtype == wl.d_dtype:
-            line["fused_adamw_exchange"] = time_fused_adamw(wl, min(args.steps, 10), exchange=True)
+            line["fused_adamw_exchange"] = time_fused_adamw(wl, few, exchange=True, peak=peak, peak_kind=peak_kind)
     if world == 1 and wl.g_dtype == wl.d_dtype:
-        line["exchange_mode"] = time_exchange_mode(wl, min(args.steps, 10))
+        line["exchange_mode"] = time_exchange_mode(wl, few)
     if not args.no_e2e:
         # every rank takes the same branch: the decision to run is agreed on first, and the
         # result is reduced by all ranks whether or not a rank failed
@@ -657,27 +836,29 @@ def main():
             (bytes_per_param(g_dtype)) + (4 << 30)
         if free > need:
             wl2 = Workload(args.also, device, 1)
-            s2, p2 = time_steps(wl2, min(args.steps, 10), 3)
+            s2, p2 = time_steps(wl2, few, 3)
             r2 = check_regime(wl2)
             also = summarize(wl2, s2, p2, peak, peak_kind)
-            also.update({"workload": workload_config(args.also, wl2)["workload"],
-                         "params": wl2.params, "steps": min(args.steps, 10),
+            also.update({"workload": workload_config(args.also)["workload"],
+                         "params": wl2.params, "steps": few,
                          "value": wl2.params / (also["ms_per_step"] * 1e-3), "unit": UNIT,
                          "regime_check": {"cos": r2.cos, "regime": gb.REGIME_NAMES[r2.regime]}})
             if wl2.g_dtype == wl2.d_dtype:
-                also["exchange_mode"] = time_exchange_mode(wl2, min(args.steps, 10))
+                also["exchange_mode"] = time_exchange_mode(wl2, few)
             line["also"] = also
             wl2.close()
         else:
             line["also"] = {"skipped": f"needs {need} bytes of device memory, {free} free"}
 
+    if world == 1 and args.others != "none":
+        line["others"] = {}
+        for name in args.others.split(","):
+            if name and name != args.workload and name != args.also:
+                line["others"][name] = time_other(name, device, few, peak,
+                                                  adamw=(not args.no_adamw and name.endswith("_dbf16")))
+
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
-        probe = time_oracle(args.workload, 8_000_000, 1, 0)
-        target = int(min(1_500_000_000, max(8_000_000, probe["value"] * 6.0)))
-        first = time_oracle(args.workload, target, 1, 1)
-        passes = int(min(30, max(2, math.ceil(12.0 / max(first["seconds_per_pass"], 1e-3)))))
-        cb = time_oracle(args.workload, target, passes, 0)
-        line["cpu_baseline"] = {k: cb[k] for k in ("value", "unit", "cores", "kind", "sample")}
+        line["cpu_baseline"] = cpu_baseline(args.workload)
 
     if world > 1 or args.sharded:
         torch.distributed.barrier()

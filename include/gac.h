@@ -22,6 +22,7 @@
 #ifndef GAC_H_
 #define GAC_H_
 
+#include <stddef.h>
 #include <stdint.h>
 
 #ifdef __cplusplus
@@ -37,7 +38,8 @@ typedef enum {
     GAC_ERR_CUDA = 3,          /* a CUDA runtime call failed; message has the CUDA error     */
     GAC_ERR_STATE = 4,         /* calls out of order (project without stats, step going back)*/
     GAC_ERR_NONFINITE = 5,     /* NaN/Inf met in g or d; the step is reported as a violation  */
-    GAC_ERR_TIMEOUT = 6        /* reserved: no kernel of this library waits on a flag or a peer  */
+    GAC_ERR_TIMEOUT = 6        /* gac_decide_exchange: a peer's sums did not arrive within the limit
+                                  (the only wait in this library, bounded)                      */
 } gac_status;
 
 typedef enum { GAC_F32 = 0, GAC_BF16 = 1 } gac_dtype;
@@ -87,7 +89,9 @@ typedef struct {
                                   sends on is scaled by min(1, clip_max_norm/(norm + clip_eps)),
                                   with the norm taken in closed form from the three sums, so the
                                   separate clipping pass of the optimizer is not needed.  0 = off.
-                                  The stored direction is never clipped.                           */
+                                  The stored direction is not clipped in state modes RAW, EXCHANGE
+                                  and HOLD (it is the raw gradient, or left alone); PROJECTED stores
+                                  d' = g' as written, hence clipped.                                */
     double clip_eps;           /* 1e-6 (the usual constant of global-norm clipping)                */
 } gac_hparams;
 
@@ -118,7 +122,8 @@ typedef struct {
     uint32_t ref_lost;         /* exchange mode only: a non-finite step was closed, the stored
                                   direction is gone and the next step restarts from the zero
                                   reference (Algorithm 1's g_0 = 0)                               */
-    uint32_t reserved;
+    uint32_t timed_out;        /* peer exchange only: a rank's numbers did not arrive within the limit;
+                                  no decision was taken and the pass that follows writes nothing    */
 } gac_result;
 
 /* Fills *hp with the paper's defaults. */
@@ -169,16 +174,62 @@ int gac_stats(gac_ctx *ctx, uint64_t step, uint32_t staleness, void *cuda_stream
  * "Efficient computation under data parallelism"): each rank reduces its own
  * shard, ONE all-reduce sums three numbers, every rank takes the same decision.
  *   gac_stats_partial  writes this context's local (dot, gg, dd) to
- *                      sums_out, a DEVICE pointer to 3 doubles owned by the
- *                      caller, and takes no decision;
+ *                      sums_out, a DEVICE pointer to 3 doubles (8-byte aligned)
+ *                      owned by the caller, and takes no decision;
  *   gac_decide         reads the GLOBAL (dot, gg, dd) from sums_in (device
- *                      pointer to 3 doubles, e.g. after an all-reduce on the
- *                      same stream) and fills the decision record.
+ *                      pointer to 3 doubles, 8-byte aligned, e.g. after an
+ *                      all-reduce on the same stream) and fills the decision record.
  * The collective between the two calls is the caller's.
  */
 int gac_stats_partial(gac_ctx *ctx, uint64_t step, uint32_t staleness, void *cuda_stream,
                       double *sums_out);
 int gac_decide(gac_ctx *ctx, void *cuda_stream, const double *sums_in, gac_result *host_out);
+
+/*
+ * Peer exchange: the sharded form WITHOUT a collective library.  App. A.1 needs
+ * one all-reduce of three numbers per step and App. A.2 names it as GAC's one
+ * extra synchronisation point.  Here the kernels do it themselves:
+ *   gac_stats_exchange   reduces this rank's shard like gac_stats_partial; the
+ *                        last CTA of that same kernel then stores the three sums
+ *                        and the step number into this rank's slot of EVERY
+ *                        rank's slot array (plain stores over NVLink for a peer,
+ *                        no multicast, no bulk copy), and returns.  Nothing waits.
+ *   gac_decide_exchange  one small kernel: waits until the slots of all ranks in
+ *                        this rank's own array carry the step number, adds them
+ *                        in RANK ORDER (every rank does the same additions in the
+ *                        same order: bit-identical sums and decisions everywhere)
+ *                        and fills the decision record, as gac_decide does.
+ * Other work may be enqueued between the two calls.  The wait is bounded by the
+ * timeout given to gac_exchange_attach (wall time on the device, plus a cap on
+ * the number of polls); when it runs out the record is marked `timed_out`, no
+ * decision is taken, and a following gac_project / gac_project_adamw writes
+ * NOTHING (neither g nor d; in exchange state mode the stored direction is then
+ * lost, as after a non-finite step).  With host_out the call returns
+ * GAC_ERR_TIMEOUT and the step stays pending: gac_decide_exchange may be
+ * repeated (the posted numbers stay where they are), or the step redone with
+ * gac_stats_partial / gac_decide and the caller's own collective.
+ *
+ * gac_exchange_attach   rank, world (<= GAC_EXCHANGE_MAX_RANKS), and `slots`: a
+ *                       host array of `world` DEVICE pointers, slots[r] = rank r's
+ *                       slot array as addressable from this context's device
+ *                       (slots[rank] is this rank's own).  Every array has
+ *                       gac_exchange_bytes(world) bytes, is 32-byte aligned,
+ *                       CALLER-owned, and must be zero-filled before the first
+ *                       step and whenever step numbers start over.  How a peer's
+ *                       array becomes addressable (peer access within a process,
+ *                       an IPC or symmetric-memory mapping between processes) is
+ *                       the caller's business.  timeout_ms = 0 means 1000.
+ *                       Allocates a small table (not capturable).
+ * Each array holds two sets of slots, used by odd and even steps in turn; that
+ * is enough because a rank cannot post step t+2 before every peer has read the
+ * slots of step t (it needs the peers' numbers of step t+1 first).
+ * Errors: INVALID_ARG, STATE (not attached, calls out of order), CUDA, TIMEOUT.
+ */
+#define GAC_EXCHANGE_MAX_RANKS 1024
+size_t gac_exchange_bytes(uint32_t world);
+int gac_exchange_attach(gac_ctx *ctx, uint32_t rank, uint32_t world, void *const *slots, uint32_t timeout_ms);
+int gac_stats_exchange(gac_ctx *ctx, uint64_t step, uint32_t staleness, void *cuda_stream);
+int gac_decide_exchange(gac_ctx *ctx, void *cuda_stream, gac_result *host_out);
 
 /*
  * gac_project -- one pass that reads g and d once and writes g' and d' in
@@ -191,7 +242,8 @@ int gac_decide(gac_ctx *ctx, void *cuda_stream, const double *sums_in, gac_resul
  *                    skips its optimizer step (Algorithm 1: theta_t = theta_{t-1})
  *   every regime     d'_i = g_i, the raw gradient (state_mode RAW; EXCHANGE reaches the
  *                    same state without this copy, see "Exchange mode" below)
- *   nonfinite        neither g nor d is written
+ *   nonfinite        neither g nor d is written (the same holds for a record
+ *                    marked timed_out by gac_decide_exchange)
  * Must follow a gac_stats / gac_decide of the same step (else STATE).
  *   coef_override    host pointer to one float, or NULL.  When given, it
  *                    replaces the record's `coef` (used to compare outputs
@@ -333,13 +385,22 @@ int gac_get_info(const gac_ctx *ctx, gac_info *out);
  *                    pointers, caller-owned, only read)
  *   cuda_device      device that owns g, d and result_dev (0..63)
  *   cuda_stream      stream for the two small copies and the one kernel launch
- *   result_dev       DEVICE pointer, caller-owned: receives the gac_result of
- *                    this step when the stream reaches that point.  Nothing is
- *                    copied to the host and the call does not synchronise.
+ *   result_dev       DEVICE pointer, caller-owned, 8-byte aligned: receives the
+ *                    gac_result of this step when the stream reaches that point
+ *                    (every field is written; applied_steps and ref_lost read 0).
+ *                    Nothing is copied back to the host.
+ *
+ * Host-side behaviour: the chunk table is copied to the device from ordinary
+ * (pageable) library memory.  Such a copy makes the calling thread wait until
+ * the work queued earlier on cuda_stream has drained and the table has been
+ * staged; the reduction itself then runs asynchronously.  A caller that cannot
+ * afford that wait gives the call a stream of its own and orders it with events.
  *
  * The first call on each device looks up the device address of the built-in
- * array (once, with that device current); make that first call outside any
- * stream capture.  Later calls reuse the address.
+ * array (once, with that device current).  No call may be made on a stream that
+ * is being captured into a CUDA graph: a replay would copy the table from the
+ * library's host buffer as it stands THEN, after other calls have rewritten it.
+ * Such a call is refused with GAC_ERR_STATE and nothing is enqueued.
  *
  * All calls on a device share the one array, and it keeps what the previous
  * call left: each call re-zeroes the ticket and rewrites the table on its
@@ -347,7 +408,8 @@ int gac_get_info(const gac_ctx *ctx, gac_info *out);
  * streams without ordering, or two host threads) race on that array and give
  * wrong sums: order them on one stream or with events.
  * Only the statistics pass has this form; gac_project still wants a context.
- * Errors: INVALID_ARG, DTYPE, CUDA (message via gac_last_error(NULL)).
+ * Errors: INVALID_ARG, DTYPE, STATE (stream is capturing), CUDA (message via
+ * gac_last_error(NULL)).
  */
 #define GAC_STATIC_MAX_CHUNKS 65536
 #define GAC_STATIC_SCRATCH_BYTES (256 + 62976 + GAC_STATIC_MAX_CHUNKS * 32)

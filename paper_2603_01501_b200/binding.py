@@ -46,7 +46,7 @@ class gac_result(ctypes.Structure):
                 ("out_norm", ctypes.c_double), ("clip_scale", ctypes.c_double),
                 ("applied_steps", ctypes.c_uint64), ("g_set", ctypes.c_uint32),
                 ("out_set", ctypes.c_uint32), ("ref_lost", ctypes.c_uint32),
-                ("reserved", ctypes.c_uint32)]
+                ("timed_out", ctypes.c_uint32)]
 
     def as_dict(self):
         return {k: getattr(self, k) for k, _ in self._fields_}
@@ -72,7 +72,8 @@ class gac_info(ctypes.Structure):
 EXPORTS = ["gac_default_hparams", "gac_init", "gac_stats", "gac_stats_partial", "gac_decide",
            "gac_project", "gac_free", "gac_last_error", "gac_set_launch", "gac_get_info",
            "gac_stats_static", "gac_default_adamw", "gac_attach_adamw", "gac_project_adamw",
-           "gac_rebind", "gac_next_gradient_set"]
+           "gac_rebind", "gac_next_gradient_set", "gac_exchange_bytes", "gac_exchange_attach",
+           "gac_stats_exchange", "gac_decide_exchange"]
 
 _lib = None
 
@@ -121,6 +122,14 @@ def load_library() -> ctypes.CDLL:
     L.gac_project_adamw.argtypes = [vp, vp, ctypes.POINTER(gac_adamw), ctypes.POINTER(ctypes.c_float),
                                     ctypes.POINTER(gac_result)]
     L.gac_project_adamw.restype = i32
+    L.gac_exchange_bytes.argtypes = [u32]
+    L.gac_exchange_bytes.restype = ctypes.c_size_t
+    L.gac_exchange_attach.argtypes = [vp, u32, u32, ctypes.POINTER(vp), u32]
+    L.gac_exchange_attach.restype = i32
+    L.gac_stats_exchange.argtypes = [vp, u64, u32, vp]
+    L.gac_stats_exchange.restype = i32
+    L.gac_decide_exchange.argtypes = [vp, vp, ctypes.POINTER(gac_result)]
+    L.gac_decide_exchange.restype = i32
     for name in ("gac_init", "gac_stats", "gac_stats_partial", "gac_decide", "gac_project",
                  "gac_free", "gac_set_launch", "gac_get_info"):
         getattr(L, name).restype = i32
@@ -236,6 +245,41 @@ def gac_decide(ctx: GacContext, sums_in: torch.Tensor, stream=None,
     res = gac_result() if fetch else None
     rc = load_library().gac_decide(ctx.handle, _stream_ptr(stream), sums_in.data_ptr(),
                                    ctypes.byref(res) if fetch else None)
+    ctx._check(rc, allow_nonfinite=True)
+    return res
+
+
+def gac_exchange_bytes(world: int) -> int:
+    """Size of one rank's slot array for the peer exchange of the three sums."""
+    return int(load_library().gac_exchange_bytes(world))
+
+
+def gac_exchange_attach(ctx: GacContext, rank: int, world: int, slots: Sequence[torch.Tensor],
+                        timeout_ms: int = 0) -> None:
+    """gac_exchange_attach: `slots[r]` is rank r's slot array (a zero-filled CUDA uint8 tensor of
+    gac_exchange_bytes(world) bytes, or an integer device address of one mapped from a peer)."""
+    arr = (ctypes.c_void_p * max(world, 1))()
+    for r, t in enumerate(slots):
+        if isinstance(t, torch.Tensor):
+            if not (t.is_cuda and t.is_contiguous() and t.numel() * t.element_size() >= gac_exchange_bytes(world)):
+                raise ValueError("a slot array must be a contiguous CUDA tensor of gac_exchange_bytes(world) bytes")
+            arr[r] = t.data_ptr()
+        else:
+            arr[r] = int(t)
+    if len(slots) != world:
+        raise ValueError("one slot array per rank")
+    ctx._check(load_library().gac_exchange_attach(ctx.handle, rank, world, arr, timeout_ms))
+    ctx._keep_slots = list(slots)
+
+
+def gac_stats_exchange(ctx: GacContext, step: int, staleness: int = 0, stream=None) -> None:
+    ctx._check(load_library().gac_stats_exchange(ctx.handle, step, staleness, _stream_ptr(stream)))
+
+
+def gac_decide_exchange(ctx: GacContext, stream=None, fetch: bool = True) -> Optional[gac_result]:
+    """gac_decide_exchange; raises GacError(GAC_ERR_TIMEOUT) when fetching a record whose wait ran out."""
+    res = gac_result() if fetch else None
+    rc = load_library().gac_decide_exchange(ctx.handle, _stream_ptr(stream), ctypes.byref(res) if fetch else None)
     ctx._check(rc, allow_nonfinite=True)
     return res
 

@@ -13,7 +13,7 @@ KERNELS = os.path.join(HERE, "csrc", "gac_kernels.cuh")
 LIB = os.path.join(HERE, "libgac_b200.so")
 
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
-              "-Xcompiler", "-fPIC", "-shared", "-cudart", "static"]
+              "-Xcompiler", "-fPIC", "-shared", "-cudart", "static", "-ldl"]
 
 
 def build(force: bool = False, verbose: bool = False) -> str:

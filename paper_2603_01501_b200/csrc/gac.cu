@@ -17,6 +17,7 @@
 // here, hence no tensor-core path.
 #include <cuda_runtime.h>
 #include <math.h>
+#include <nvtx3/nvToolsExt.h>
 #include <stdint.h>
 #include <stdio.h>
 #include <string.h>
@@ -61,6 +62,12 @@ struct gac_ctx {
     int grid_stats = 0, grid_project = 0;
     int threads_stats = 0, threads_project = 0;
     const void *project_fn = nullptr;   // instantiation chosen from the hyper-parameters
+    // peer exchange of the three sums (gac_exchange_attach)
+    uint32_t xchg_world = 0, xchg_rank = 0;
+    unsigned long long *d_peers = nullptr;   // device table of every rank's slot array, as addressable from this GPU
+    PeerSlot *xchg_slots = nullptr;          // this rank's own slot array (caller-owned)
+    unsigned long long xchg_timeout_ns = 0;
+    bool posted = false;                     // the pending partial reduction was posted to the peers
     OptChunk *d_opt_chunks = nullptr;   // optimizer state table of gac_attach_adamw
     std::vector<gac_opt_tensor> opt_list;
     int grid_adamw = 0, threads_adamw = 0;
@@ -108,10 +115,19 @@ struct DeviceGuard {
 
 size_t elem_size(int dt) { return dt == GAC_BF16 ? 2 : 4; }
 
+// Named range around the host side of a call, visible in a timeline profiler; costs one
+// pointer test when no tool is attached.
+struct Range {
+    explicit Range(const char *name) { nvtxRangePushA(name); }
+    ~Range() { nvtxRangePop(); }
+};
+
 void release_device(gac_ctx *c) {
     if (c->d_chunks) cudaFree(c->d_chunks);
     if (c->d_opt_chunks) cudaFree(c->d_opt_chunks);
     c->d_opt_chunks = nullptr;
+    if (c->d_peers) cudaFree(c->d_peers);
+    c->d_peers = nullptr;
     if (c->d_partials) cudaFree(c->d_partials);
     if (c->d_ticket) cudaFree(c->d_ticket);
     if (c->d_rec) cudaFree(c->d_rec);
@@ -312,8 +328,11 @@ int check_list(gac_ctx *ctx, const gac_tensor *list, uint32_t n, size_t gs, size
     return GAC_OK;
 }
 
-DevHP dev_hp(const gac_ctx *c, uint64_t step, uint32_t staleness, int decide) {
+DevHP dev_hp(const gac_ctx *c, uint64_t step, uint32_t staleness, int decide, bool exchange = false) {
     DevHP h;
+    h.xchg_world = exchange ? c->xchg_world : 0u;
+    h.xchg_rank = c->xchg_rank;
+    h.xchg_peers = c->d_peers;
     h.c_low = c->hp.c_low;
     h.c_high = c->hp.c_high;
     h.eps = c->hp.eps;
@@ -336,17 +355,20 @@ int read_back(gac_ctx *c, cudaStream_t s, gac_result *host_out) {
     GAC_CUDA(c, cudaMemcpyAsync(c->h_rec, c->d_rec, sizeof(gac_result), cudaMemcpyDeviceToHost, s));
     GAC_CUDA(c, cudaStreamSynchronize(s));
     *host_out = *c->h_rec;
+    if (host_out->timed_out)
+        return fail(c, GAC_ERR_TIMEOUT, "the sums of step %s%lld did not arrive from every rank within the limit", "",
+                    (long long)host_out->step);
     if (host_out->nonfinite)
         return fail(c, GAC_ERR_NONFINITE, "NaN or Inf met in the gradient or the stored direction%s");
     return GAC_OK;
 }
 
 int launch_stats(gac_ctx *c, uint64_t step, uint32_t staleness, cudaStream_t s, double *sums_out,
-                 int decide) {
+                 int decide, bool exchange = false) {
     if (step == 0) return fail(c, GAC_ERR_INVALID_ARG, "step counts from 1 (Algorithm 1)%s");
     if (c->started && step <= c->last_projected_step)
         return fail(c, GAC_ERR_STATE, "step %s%lld was already projected", "", (long long)step);
-    const DevHP h = dev_hp(c, step, staleness, decide);
+    const DevHP h = dev_hp(c, step, staleness, decide, exchange);
     const uint32_t nc = uint32_t(c->n_chunks);
     stats_kernel_of(c->pair)<<<c->grid_stats, c->threads_stats, 0, s>>>(c->d_chunks, nc, c->d_partials, c->d_ticket,
                                                                         c->d_rec, sums_out, h);
@@ -460,23 +482,29 @@ int gac_rebind(gac_ctx *ctx, const gac_tensor *list, uint32_t n) {
 
 int gac_stats(gac_ctx *ctx, uint64_t step, uint32_t staleness, void *cuda_stream, gac_result *host_out) {
     if (!ctx) return fail(nullptr, GAC_ERR_INVALID_ARG, "ctx is NULL%s");
+    Range range("gac_stats");
     DeviceGuard guard(ctx->device);
     cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
     if (int rc = launch_stats(ctx, step, staleness, s, nullptr, 1)) return rc;
     ctx->started = true;
     ctx->stats_pending = false;
+    ctx->posted = false;
     ctx->decision_ready = true;
     return host_out ? read_back(ctx, s, host_out) : GAC_OK;
 }
 
 int gac_stats_partial(gac_ctx *ctx, uint64_t step, uint32_t staleness, void *cuda_stream, double *sums_out) {
     if (!ctx) return fail(nullptr, GAC_ERR_INVALID_ARG, "ctx is NULL%s");
+    Range range("gac_stats_partial");
     if (!sums_out) return fail(ctx, GAC_ERR_INVALID_ARG, "sums_out is NULL%s");
+    if (reinterpret_cast<uint64_t>(sums_out) % 8)
+        return fail(ctx, GAC_ERR_INVALID_ARG, "sums_out must be 8-byte aligned (three doubles)%s");
     DeviceGuard guard(ctx->device);
     cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
     if (int rc = launch_stats(ctx, step, staleness, s, sums_out, 0)) return rc;
     ctx->started = true;
     ctx->stats_pending = true;
+    ctx->posted = false;
     ctx->decision_ready = false;
     ctx->pending_staleness = staleness;
     return GAC_OK;
@@ -484,8 +512,12 @@ int gac_stats_partial(gac_ctx *ctx, uint64_t step, uint32_t staleness, void *cud
 
 int gac_decide(gac_ctx *ctx, void *cuda_stream, const double *sums_in, gac_result *host_out) {
     if (!ctx) return fail(nullptr, GAC_ERR_INVALID_ARG, "ctx is NULL%s");
+    Range range("gac_decide");
     if (!sums_in) return fail(ctx, GAC_ERR_INVALID_ARG, "sums_in is NULL%s");
-    if (!ctx->stats_pending) return fail(ctx, GAC_ERR_STATE, "gac_decide needs a gac_stats_partial first%s");
+    if (reinterpret_cast<uint64_t>(sums_in) % 8)
+        return fail(ctx, GAC_ERR_INVALID_ARG, "sums_in must be 8-byte aligned (three doubles)%s");
+    if (!ctx->stats_pending || ctx->posted)
+        return fail(ctx, GAC_ERR_STATE, "gac_decide needs a gac_stats_partial first%s");
     DeviceGuard guard(ctx->device);
     cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
     const DevHP h = dev_hp(ctx, ctx->pending_step, ctx->pending_staleness, 1);
@@ -497,8 +529,80 @@ int gac_decide(gac_ctx *ctx, void *cuda_stream, const double *sums_in, gac_resul
     return host_out ? read_back(ctx, s, host_out) : GAC_OK;
 }
 
+size_t gac_exchange_bytes(uint32_t world) { return size_t(world) * 2 * sizeof(PeerSlot); }
+
+int gac_exchange_attach(gac_ctx *ctx, uint32_t rank, uint32_t world, void *const *slots, uint32_t timeout_ms) {
+    if (!ctx) return fail(nullptr, GAC_ERR_INVALID_ARG, "ctx is NULL%s");
+    if (world == 0 || world > GAC_EXCHANGE_MAX_RANKS || rank >= world)
+        return fail(ctx, GAC_ERR_INVALID_ARG, "peer exchange needs 1 <= world <= %s%lld and rank < world", "",
+                    (long long)GAC_EXCHANGE_MAX_RANKS);
+    if (!slots) return fail(ctx, GAC_ERR_INVALID_ARG, "slots is NULL%s");
+    if (ctx->stats_pending || ctx->decision_ready)
+        return fail(ctx, GAC_ERR_STATE, "gac_exchange_attach between the calls of a step would split it%s");
+    std::vector<unsigned long long> table(world);
+    for (uint32_t r = 0; r < world; ++r) {
+        const uint64_t a = reinterpret_cast<uint64_t>(slots[r]);
+        if (!a || a % sizeof(PeerSlot))
+            return fail(ctx, GAC_ERR_INVALID_ARG, "slot array of rank %s%lld is NULL or not 32-byte aligned", "", r);
+        table[r] = a;
+    }
+    DeviceGuard guard(ctx->device);
+    if (ctx->d_peers) {
+        cudaFree(ctx->d_peers);
+        ctx->d_peers = nullptr;
+    }
+    GAC_CUDA(ctx, cudaMalloc(&ctx->d_peers, world * sizeof(unsigned long long)));
+    GAC_CUDA(ctx, cudaMemcpy(ctx->d_peers, table.data(), world * sizeof(unsigned long long), cudaMemcpyHostToDevice));
+    ctx->xchg_world = world;
+    ctx->xchg_rank = rank;
+    ctx->xchg_slots = static_cast<PeerSlot *>(slots[rank]);
+    ctx->xchg_timeout_ns = uint64_t(timeout_ms ? timeout_ms : 1000u) * 1000000ull;
+    return GAC_OK;
+}
+
+int gac_stats_exchange(gac_ctx *ctx, uint64_t step, uint32_t staleness, void *cuda_stream) {
+    if (!ctx) return fail(nullptr, GAC_ERR_INVALID_ARG, "ctx is NULL%s");
+    Range range("gac_stats_exchange");
+    if (!ctx->xchg_world) return fail(ctx, GAC_ERR_STATE, "gac_stats_exchange needs gac_exchange_attach first%s");
+    DeviceGuard guard(ctx->device);
+    cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+    if (int rc = launch_stats(ctx, step, staleness, s, nullptr, 0, true)) return rc;
+    ctx->started = true;
+    ctx->stats_pending = true;
+    ctx->posted = true;
+    ctx->decision_ready = false;
+    ctx->pending_staleness = staleness;
+    return GAC_OK;
+}
+
+int gac_decide_exchange(gac_ctx *ctx, void *cuda_stream, gac_result *host_out) {
+    if (!ctx) return fail(nullptr, GAC_ERR_INVALID_ARG, "ctx is NULL%s");
+    Range range("gac_decide_exchange");
+    if (!ctx->stats_pending || !ctx->posted)
+        return fail(ctx, GAC_ERR_STATE, "gac_decide_exchange needs a gac_stats_exchange first%s");
+    DeviceGuard guard(ctx->device);
+    cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+    const DevHP h = dev_hp(ctx, ctx->pending_step, ctx->pending_staleness, 1, true);
+    gac_decide_exchange_kernel<<<1, kExchangeThreads, 0, s>>>(ctx->xchg_slots, ctx->d_rec, h, ctx->xchg_timeout_ns);
+    GAC_CUDA(ctx, cudaGetLastError());
+    ++ctx->launches;
+    if (host_out) {
+        const int rc = read_back(ctx, s, host_out);
+        if (rc == GAC_ERR_TIMEOUT) return rc;   // still pending: the call may be repeated once the peers have posted
+        ctx->stats_pending = false;
+        ctx->posted = false;
+        ctx->decision_ready = true;
+        return rc;
+    }
+    ctx->stats_pending = false;
+    ctx->posted = false;
+    ctx->decision_ready = true;
+    return GAC_OK;
+}
+
 int gac_project(gac_ctx *ctx, void *cuda_stream, const float *coef_override, gac_result *host_out) {
     if (!ctx) return fail(nullptr, GAC_ERR_INVALID_ARG, "ctx is NULL%s");
+    Range range("gac_project");
     if (!ctx->decision_ready)
         return fail(ctx, GAC_ERR_STATE, "gac_project needs the decision of gac_stats / gac_decide for this step%s");
     DeviceGuard guard(ctx->device);
@@ -550,6 +654,7 @@ int gac_attach_adamw(gac_ctx *ctx, const gac_opt_tensor *list, uint32_t n, uint6
 int gac_project_adamw(gac_ctx *ctx, void *cuda_stream, const gac_adamw *opt, const float *coef_override,
                       gac_result *host_out) {
     if (!ctx) return fail(nullptr, GAC_ERR_INVALID_ARG, "ctx is NULL%s");
+    Range range("gac_project_adamw");
     if (!opt) return fail(ctx, GAC_ERR_INVALID_ARG, "opt is NULL%s");
     if (!ctx->d_opt_chunks) return fail(ctx, GAC_ERR_STATE, "gac_project_adamw needs gac_attach_adamw first%s");
     if (!ctx->decision_ready)
@@ -563,7 +668,8 @@ int gac_project_adamw(gac_ctx *ctx, void *cuda_stream, const gac_adamw *opt, con
     const float k = coef_override ? *coef_override : 0.0f;
     const int use = coef_override ? 1 : 0;
     const uint32_t nc = uint32_t(ctx->n_chunks);
-    const AdamDev o{opt->lr, opt->beta1, opt->beta2, opt->eps, opt->weight_decay};
+    const AdamDev o{opt->lr, opt->beta1, opt->beta2, opt->eps, 1.0 - opt->beta1, 1.0 - opt->beta2,
+                    opt->lr * opt->weight_decay};
     const bool exch = (ctx->hp.state_mode == GAC_STATE_EXCHANGE);
     const AdamKernel ak = with_pair(ctx->pair, [exch](auto tag) -> AdamKernel {
         return exch ? gac_adamw_kernel<decltype(tag), true> : gac_adamw_kernel<decltype(tag), false>;
@@ -677,6 +783,8 @@ extern "C" int gac_stats_static(const gac_tensor *list, uint32_t n, int g_dtype,
     if (!list || n == 0) return fail(nullptr, GAC_ERR_INVALID_ARG, "empty tensor list%s");
     if (!hp) return fail(nullptr, GAC_ERR_INVALID_ARG, "hp is NULL%s");
     if (!result_dev) return fail(nullptr, GAC_ERR_INVALID_ARG, "result_dev is NULL%s");
+    if (reinterpret_cast<uint64_t>(result_dev) % 8)
+        return fail(nullptr, GAC_ERR_INVALID_ARG, "result_dev must be 8-byte aligned (a gac_result holds doubles)%s");
     if (step == 0) return fail(nullptr, GAC_ERR_INVALID_ARG, "step counts from 1 (Algorithm 1)%s");
     if (pair_id(g_dtype, d_dtype) < 0)
         return fail(nullptr, GAC_ERR_DTYPE, "supported (g,d) element types: (f32,f32), (bf16,f32), (bf16,bf16)%s");
@@ -704,13 +812,23 @@ extern "C" int gac_stats_static(const gac_tensor *list, uint32_t n, int g_dtype,
 
     DeviceGuard guard(cuda_device);
     if (!guard.ok) return fail(nullptr, GAC_ERR_CUDA, "cudaSetDevice failed%s");
+    cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+    {
+        // A captured copy node would read the library's shared host table when the graph is
+        // replayed, after other calls have refilled it: refuse instead of replaying a stale table.
+        cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
+        GAC_CUDA(nullptr, cudaStreamIsCapturing(s, &cap));
+        if (cap != cudaStreamCaptureStatusNone)
+            return fail(nullptr, GAC_ERR_STATE,
+                        "gac_stats_static cannot be captured in a CUDA graph: its table copy reads a host buffer "
+                        "that every call rewrites%s");
+    }
     StaticSetup *st = nullptr;
     if (int rc = static_setup(cuda_device, &st)) return rc;
 
     // Host-side image of the table in a fixed buffer of the library (no heap use either), then one
     // copy into the device scratch.  The lock covers filling and staging: the copy call returns once
     // the pageable source has been staged, after which the buffer may be refilled by another caller.
-    cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
     Chunk *d_chunks = reinterpret_cast<Chunk *>(st->base + kStaticChunksOff);
     double *d_partials = reinterpret_cast<double *>(st->base + kStaticPartialsOff);
     unsigned *d_ticket = reinterpret_cast<unsigned *>(st->base + kStaticTicketOff);
@@ -731,6 +849,9 @@ extern "C" int gac_stats_static(const gac_tensor *list, uint32_t n, int g_dtype,
         }
         // the scratch keeps whatever the previous call left: the ticket must start at zero
         GAC_CUDA(nullptr, cudaMemsetAsync(d_ticket, 0, sizeof(unsigned), s));
+        // the caller's record may hold anything: fields the reduction does not write (applied_steps,
+        // ref_lost) read as zero afterwards
+        GAC_CUDA(nullptr, cudaMemsetAsync(result_dev, 0, sizeof(gac_result), s));
         GAC_CUDA(nullptr, cudaMemcpyAsync(d_chunks, g_static_host_table, filled * sizeof(Chunk),
                                           cudaMemcpyHostToDevice, s));
     }

@@ -51,7 +51,21 @@ struct DevHP {
     int decide;      // 0: only publish the three sums (sharded form)
     double clip_max, clip_eps;
     int swapped;     // exchange mode: 1 when the table's d addresses hold this step's gradient
+    // peer exchange of the three sums (sharded form without a collective library): 0 ranks = off
+    unsigned xchg_world, xchg_rank;
+    const unsigned long long *xchg_peers;   // device table: address of every rank's slot array, as seen from this GPU
 };
+
+// One rank's contribution to one step, as it lies in a slot array: 32 bytes, the flag last.
+struct __align__(32) PeerSlot {
+    double dot, gg, dd;
+    unsigned long long step;   // Algorithm 1's t for which the three numbers hold; 0 = never written
+};
+// A slot array holds two sets of `world` slots, used by odd and even steps in turn: a rank can
+// be at most one step ahead of a peer that has not yet read the previous step's slots.
+__device__ __forceinline__ size_t peer_slot_index(unsigned long long step, unsigned world, unsigned rank) {
+    return size_t(step & 1ull) * world + rank;
+}
 
 struct F4 {
     float x, y, z, w;
@@ -79,16 +93,26 @@ __device__ __forceinline__ void st_vec(V *p, V v) {
 template <typename GT>
 struct Elem;
 
+// Raw = four elements as they lie in memory (what a thread keeps in registers
+// while loads are in flight); unpack/pack convert to and from four binary32 values.
 template <>
 struct Elem<float> {
+    using Raw = float4;
+    static __device__ __forceinline__ Raw zero() { return make_float4(0.f, 0.f, 0.f, 0.f); }
+    template <int LD>
+    static __device__ __forceinline__ Raw load_raw(const void *base, uint32_t v) {
+        return ld_vec<LD>(reinterpret_cast<const float4 *>(base) + v);
+    }
+    static __device__ __forceinline__ void store_raw(void *base, uint32_t v, Raw r) {
+        st_vec(reinterpret_cast<float4 *>(base) + v, r);
+    }
+    static __device__ __forceinline__ F4 unpack(Raw t) { return F4{t.x, t.y, t.z, t.w}; }
+    static __device__ __forceinline__ Raw pack(F4 a) { return make_float4(a.x, a.y, a.z, a.w); }
     template <int LD>
     static __device__ __forceinline__ F4 load4(const void *base, uint32_t v) {
-        float4 t = ld_vec<LD>(reinterpret_cast<const float4 *>(base) + v);
-        return F4{t.x, t.y, t.z, t.w};
+        return unpack(load_raw<LD>(base, v));
     }
-    static __device__ __forceinline__ void store4(void *base, uint32_t v, F4 a) {
-        st_vec(reinterpret_cast<float4 *>(base) + v, make_float4(a.x, a.y, a.z, a.w));
-    }
+    static __device__ __forceinline__ void store4(void *base, uint32_t v, F4 a) { store_raw(base, v, pack(a)); }
     static __device__ __forceinline__ float load1(const void *base, uint32_t i) {
         return reinterpret_cast<const float *>(base)[i];
     }
@@ -153,9 +177,9 @@ template <> struct ProjGeom<bf16_pair_t>  { static constexpr int T = 512, U = 8,
 template <> struct ExchGeom<float>        { static constexpr int T = 512, U = 4, UK = 8, C = 1, MINB = 1; };
 template <> struct ExchGeom<bf16_t>       { static constexpr int T = 512, U = 4, UK = 8, C = 1, MINB = 1; };   // pair not served
 template <> struct ExchGeom<bf16_pair_t>  { static constexpr int T = 512, U = 4, UK = 8, C = 2, MINB = 2; };
-template <> struct AdamGeom<float>        { static constexpr int T = 1024, U = 1, C = 1; };
-template <> struct AdamGeom<bf16_t>       { static constexpr int T = 1024, U = 1, C = 1; };
-template <> struct AdamGeom<bf16_pair_t>  { static constexpr int T = 1024, U = 1, C = 1; };
+template <> struct AdamGeom<float>        { static constexpr int T = 896, U = 1, C = 1; };
+template <> struct AdamGeom<bf16_t>       { static constexpr int T = 640, U = 1, C = 1; };
+template <> struct AdamGeom<bf16_pair_t>  { static constexpr int T = 640, U = 1, C = 1; };
 #endif
 
 __device__ __forceinline__ uint32_t pack_bf16x2_rn(float lo, float hi) {
@@ -166,16 +190,27 @@ __device__ __forceinline__ uint32_t pack_bf16x2_rn(float lo, float hi) {
 
 template <>
 struct Elem<bf16_t> {
+    using Raw = uint2;   // four bfloat16 values stay packed (two registers) until they are used
+    static __device__ __forceinline__ Raw zero() { return make_uint2(0u, 0u); }
     template <int LD>
-    static __device__ __forceinline__ F4 load4(const void *base, uint32_t v) {
-        uint2 t = ld_vec<LD>(reinterpret_cast<const uint2 *>(base) + v);
+    static __device__ __forceinline__ Raw load_raw(const void *base, uint32_t v) {
+        return ld_vec<LD>(reinterpret_cast<const uint2 *>(base) + v);
+    }
+    static __device__ __forceinline__ void store_raw(void *base, uint32_t v, Raw r) {
+        st_vec(reinterpret_cast<uint2 *>(base) + v, r);
+    }
+    static __device__ __forceinline__ F4 unpack(Raw t) {
         return F4{__uint_as_float(t.x << 16), __uint_as_float(t.x & 0xFFFF0000u),
                   __uint_as_float(t.y << 16), __uint_as_float(t.y & 0xFFFF0000u)};
     }
-    static __device__ __forceinline__ void store4(void *base, uint32_t v, F4 a) {
-        st_vec(reinterpret_cast<uint2 *>(base) + v,
-               make_uint2(pack_bf16x2_rn(a.x, a.y), pack_bf16x2_rn(a.z, a.w)));
+    static __device__ __forceinline__ Raw pack(F4 a) {
+        return make_uint2(pack_bf16x2_rn(a.x, a.y), pack_bf16x2_rn(a.z, a.w));
     }
+    template <int LD>
+    static __device__ __forceinline__ F4 load4(const void *base, uint32_t v) {
+        return unpack(load_raw<LD>(base, v));
+    }
+    static __device__ __forceinline__ void store4(void *base, uint32_t v, F4 a) { store_raw(base, v, pack(a)); }
     static __device__ __forceinline__ float load1(const void *base, uint32_t i) {
         return __uint_as_float(uint32_t(reinterpret_cast<const uint16_t *>(base)[i]) << 16);
     }
@@ -279,8 +314,7 @@ __device__ void take_decision(double dot, double gg, double dd, const DevHP &hp,
     r->step = hp.step;
     r->g_set = uint32_t(hp.swapped);
     r->out_set = r->g_set;
-    r->ref_lost = 0u;
-    r->reserved = 0u;
+    r->timed_out = 0u;   // ref_lost is not touched here: the pass that closes the step owns it
     r->nonfinite = !(isfinite(dot) && isfinite(gg) && isfinite(dd));
     if (r->nonfinite) {
         r->cos = __longlong_as_double(0x7FF8000000000000LL);
@@ -341,22 +375,23 @@ __device__ __forceinline__ void stats_chunk(const Chunk &ch, double &a_dot, doub
     if (ch.flags & kChunkAligned) {
         const uint32_t nvec = ch.n >> 2;
         for (uint32_t base = 0; base < nvec; base += T * U) {
-            F4 gv[U], dv[U];
+            typename Elem<GOf<GT>>::Raw gr[U];
+            typename Elem<DOf<GT>>::Raw dr[U];
 #pragma unroll
             for (int u = 0; u < U; ++u) {
                 const uint32_t v = base + u * T + tid;
+                gr[u] = Elem<GOf<GT>>::zero();
+                dr[u] = Elem<DOf<GT>>::zero();
                 if (v < nvec) {
-                    gv[u] = Elem<GOf<GT>>::template load4<GAC_LD_STATS>(g, v);
-                    if (READ_D) dv[u] = Elem<DOf<GT>>::template load4<GAC_LD_STATS>(d, v);
-                } else {
-                    gv[u] = F4{0.f, 0.f, 0.f, 0.f};
-                    if (READ_D) dv[u] = F4{0.f, 0.f, 0.f, 0.f};
+                    gr[u] = Elem<GOf<GT>>::template load_raw<GAC_LD_STATS>(g, v);
+                    if (READ_D) dr[u] = Elem<DOf<GT>>::template load_raw<GAC_LD_STATS>(d, v);
                 }
             }
 #pragma unroll
             for (int u = 0; u < U; ++u) {
-                const float ge[4] = {gv[u].x, gv[u].y, gv[u].z, gv[u].w};
-                const float de[4] = {dv[u].x, dv[u].y, dv[u].z, dv[u].w};
+                const F4 gq = Elem<GOf<GT>>::unpack(gr[u]), dq = Elem<DOf<GT>>::unpack(dr[u]);
+                const float ge[4] = {gq.x, gq.y, gq.z, gq.w};
+                const float de[4] = {dq.x, dq.y, dq.z, dq.w};
 #pragma unroll
                 for (int e = 0; e < 4; ++e) {
                     const double x = double(ge[e]);
@@ -444,6 +479,23 @@ gac_stats_kernel(const Chunk *__restrict__ chunks, uint32_t n_chunks, double *pa
             sums_out[1] = s1;
             sums_out[2] = zero_reference ? 0.0 : s2;
         }
+        if (hp.xchg_world) {
+            // App. A.1's one collective, done here: this rank's three numbers go into its slot of
+            // EVERY rank's slot array (its own included) with plain stores, then -- after a
+            // system-wide fence -- the step number that marks them valid.  Nothing is waited for.
+            const size_t idx = peer_slot_index(hp.step, hp.xchg_world, hp.xchg_rank);
+            for (unsigned r = 0; r < hp.xchg_world; ++r) {
+                volatile PeerSlot *slot = reinterpret_cast<volatile PeerSlot *>(hp.xchg_peers[r]) + idx;
+                slot->dot = zero_reference ? 0.0 : s0;
+                slot->gg = s1;
+                slot->dd = zero_reference ? 0.0 : s2;
+            }
+            __threadfence_system();
+            for (unsigned r = 0; r < hp.xchg_world; ++r) {
+                volatile PeerSlot *slot = reinterpret_cast<volatile PeerSlot *>(hp.xchg_peers[r]) + idx;
+                slot->step = hp.step;
+            }
+        }
         if (hp.decide) take_decision(s0, s1, s2, hp, zero_reference, rec);
     }
 }
@@ -453,9 +505,61 @@ __global__ void gac_decide_kernel(const double *sums_in, gac_result *rec, DevHP 
         take_decision(sums_in[0], sums_in[1], sums_in[2], hp, hp.first_step != 0, rec);
 }
 
+__device__ __forceinline__ unsigned long long global_ns() {
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+    return t;
+}
+
+// Second half of the peer exchange: thread r waits until rank r's slot of THIS rank's array
+// carries the step number, then thread 0 adds the slots in rank order -- every rank performs
+// the same additions in the same order, so all hold bit-identical sums -- and takes the
+// decision.  The wait is bounded twice (wall time and iterations); when it runs out the record
+// is marked timed_out, no decision is taken, and the pass that follows writes nothing.
+constexpr int kExchangeThreads = 128;
+__global__ void __launch_bounds__(kExchangeThreads, 1)
+gac_decide_exchange_kernel(const PeerSlot *slots, gac_result *rec, DevHP hp, unsigned long long timeout_ns) {
+    __shared__ int missing;
+    if (threadIdx.x == 0) missing = 0;
+    __syncthreads();
+    const PeerSlot *mine = slots + size_t(hp.step & 1ull) * hp.xchg_world;
+    for (unsigned r = threadIdx.x; r < hp.xchg_world; r += kExchangeThreads) {
+        const volatile unsigned long long *flag = &mine[r].step;
+        const unsigned long long t0 = global_ns();
+        const unsigned long long max_polls = timeout_ns / 64ull + 1024ull;   // second bound, should the timer stand still
+        bool there = false;
+        for (unsigned long long poll = 0; poll < max_polls; ++poll) {
+            if (*flag == hp.step) {
+                there = true;
+                break;
+            }
+            if (global_ns() - t0 > timeout_ns) break;
+            __nanosleep(256);
+        }
+        if (!there) atomicAdd(&missing, 1);
+    }
+    __syncthreads();
+    if (threadIdx.x != 0) return;
+    if (missing) {
+        rec->timed_out = 1u;
+        rec->step = hp.step;
+        return;
+    }
+    __threadfence_system();   // the flags were seen: now the numbers they guard
+    double s0 = 0.0, s1 = 0.0, s2 = 0.0;
+    for (unsigned r = 0; r < hp.xchg_world; ++r) {
+        const volatile PeerSlot *slot = mine + r;
+        s0 += slot->dot;
+        s1 += slot->gg;
+        s2 += slot->dd;
+    }
+    // the posted numbers already carry the zero reference where it applies
+    take_decision(s0, s1, s2, hp, false, rec);
+}
+
 // ----------------------------------------------------------- project kernel
 
-enum GOp { G_KEEP = 0, G_FMA = 1, G_ZERO = 2, G_SCALE = 3 };
+enum GOp { G_KEEP = 0, G_FMA = 1, G_ZERO = 2, G_SCALE = 3, G_FMA1 = 4 };   // G_FMA1: beta = 1 and no clip factor
 enum DOp { D_KEEP = 0, D_RAW = 1, D_NEW = 2, D_OUT = 3 };   // D_OUT: the new g goes into d's buffer, g stays (exchange mode)
 
 template <bool BETA1>
@@ -478,32 +582,35 @@ __device__ __forceinline__ void project_chunk(const Chunk &ch, float k, double b
     if (ch.flags & kChunkAligned) {
         const uint32_t nvec = ch.n >> 2;
         for (uint32_t base = 0; base < nvec; base += T * U) {
-            F4 gv[U], dv[U];
+            typename Elem<GOf<GT>>::Raw gr[U];
+            typename Elem<DOf<GT>>::Raw dr[U];
 #pragma unroll
             for (int u = 0; u < U; ++u) {
                 const uint32_t v = base + u * T + tid;
-                gv[u] = F4{0.f, 0.f, 0.f, 0.f};
-                dv[u] = F4{0.f, 0.f, 0.f, 0.f};
+                gr[u] = Elem<GOf<GT>>::zero();
+                dr[u] = Elem<DOf<GT>>::zero();
                 if (v < nvec) {
-                    if (kReadG) gv[u] = Elem<GOf<GT>>::template load4<GAC_LD_PROJECT>(g, v);
-                    if (kReadD) dv[u] = Elem<DOf<GT>>::template load4<GAC_LD_PROJECT>(d, v);
+                    if (kReadG) gr[u] = Elem<GOf<GT>>::template load_raw<GAC_LD_PROJECT>(g, v);
+                    if (kReadD) dr[u] = Elem<DOf<GT>>::template load_raw<GAC_LD_PROJECT>(d, v);
                 }
             }
 #pragma unroll
             for (int u = 0; u < U; ++u) {
                 const uint32_t v = base + u * T + tid;
                 if (v >= nvec) continue;
-                F4 out = gv[u];
+                const F4 gq = Elem<GOf<GT>>::unpack(gr[u]);
+                F4 out = gq;
                 if (GOP == G_ZERO) out = F4{0.f, 0.f, 0.f, 0.f};
                 if (GOP == G_FMA) {
-                    out.x = rank_one<BETA1>(gv[u].x, dv[u].x, k, beta, s);
-                    out.y = rank_one<BETA1>(gv[u].y, dv[u].y, k, beta, s);
-                    out.z = rank_one<BETA1>(gv[u].z, dv[u].z, k, beta, s);
-                    out.w = rank_one<BETA1>(gv[u].w, dv[u].w, k, beta, s);
+                    const F4 dq = Elem<DOf<GT>>::unpack(dr[u]);
+                    out.x = rank_one<BETA1>(gq.x, dq.x, k, beta, s);
+                    out.y = rank_one<BETA1>(gq.y, dq.y, k, beta, s);
+                    out.z = rank_one<BETA1>(gq.z, dq.z, k, beta, s);
+                    out.w = rank_one<BETA1>(gq.w, dq.w, k, beta, s);
                 }
-                if (GOP == G_SCALE) out = F4{scaled(gv[u].x, s), scaled(gv[u].y, s), scaled(gv[u].z, s), scaled(gv[u].w, s)};
+                if (GOP == G_SCALE) out = F4{scaled(gq.x, s), scaled(gq.y, s), scaled(gq.z, s), scaled(gq.w, s)};
                 if (GOP != G_KEEP) Elem<GOf<GT>>::store4(o, v, out);
-                if (DOP == D_RAW) Elem<DOf<GT>>::store4(d, v, gv[u]);
+                if (DOP == D_RAW) Elem<DOf<GT>>::store4(d, v, gq);
                 if (DOP == D_NEW) {
                     if (GOP == G_FMA || GOP == G_SCALE) out = Elem<GOf<GT>>::template load4<GAC_LD_PROJECT>(g, v);   // the value as stored (rounded)
                     Elem<DOf<GT>>::store4(d, v, out);
@@ -561,11 +668,12 @@ __global__ void __launch_bounds__((ProjGeomOf<GT, STATE>::T), (ProjGeomOf<GT, ST
 gac_project_kernel(const Chunk *__restrict__ chunks, uint32_t n_chunks, gac_result *rec,
                    float coef_override, int use_override, double beta, double clip_max, double clip_eps,
                    int swapped) {
-    if (rec->nonfinite) {   // reading taken for NaN/Inf: touch nothing
-        // exchange mode: the roles swap all the same, so the stored direction is gone
-        if (STATE == GAC_STATE_EXCHANGE && blockIdx.x == 0 && threadIdx.x == 0) rec->ref_lost = 1u;
-        return;
-    }
+    // Exchange mode: the roles swap whatever the step did, so a non-finite step loses the stored
+    // direction.  The flag is written here, by the pass that closes the step (never by the
+    // reduction, which may run more than once per step), and nobody reads it during this launch.
+    const bool closed = rec->nonfinite || rec->timed_out;   // no decision to act on: touch nothing
+    if (STATE == GAC_STATE_EXCHANGE && blockIdx.x == 0 && threadIdx.x == 0) rec->ref_lost = closed ? 1u : 0u;
+    if (closed) return;
     const int regime = rec->regime;
     const float k = use_override ? coef_override : rec->coef;
     constexpr int dop = STATE == GAC_STATE_RAW ? D_RAW
@@ -601,19 +709,25 @@ struct __align__(16) OptChunk {
 };
 static_assert(sizeof(OptChunk) == 32, "optimizer chunk descriptors are read as two 16-byte words");
 
+// What the host knows of the optimizer, passed by value: kernel arguments live in the constant
+// bank, where an instruction can use them as an operand without holding a register for them.
 struct AdamDev {
-    double lr, beta1, beta2, eps, weight_decay;
+    double lr, b1, b2, eps;
+    double c1, c2, lr_wd;      // 1 - b1, 1 - b2, lr * weight_decay (computed on the host, same arithmetic)
 };
 
-struct AdamConst {
-    double b1, c1, b2, c2;                       // moment recurrences
-    double step_size, inv_sqrt_bc2, eps, lr_wd;  // lr/(1-b1^t), 1/sqrt(1-b2^t), eps, lr*wd
+// What depends on the count of applied updates, which lives on the device.
+struct AdamStep {
+    double step_size, inv_sqrt_bc2;   // lr / (1 - b1^t), 1 / sqrt(1 - b2^t)
 };
 
 // The outgoing gradient in binary64, unrounded: the moments are differences of
 // nearly equal terms often enough that a binary32 g' would cost them digits.
 template <int GOP>
 __device__ __forceinline__ double outgoing64(float g, float d, float k, double beta, double s) {
+    // beta = 1, s = 1: the product of two binary32 values is exact in binary64, so this single fused
+    // operation gives the same number as the general form below
+    if (GOP == G_FMA1) return fma(double(k), double(d), double(g));
     if (GOP == G_FMA)
         return __dmul_rn(s, __dadd_rn(__dmul_rn(beta, double(g)), __dmul_rn(double(k), double(d))));
     if (GOP == G_SCALE) return __dmul_rn(s, double(g));
@@ -636,7 +750,8 @@ __device__ __forceinline__ double rcp_approx64(double x) {
     asm("rcp.approx.ftz.f64 %0, %1;" : "=d"(y) : "d"(x));
     return y;
 }
-__device__ __forceinline__ void adamw_elem(double g64, float &p, float &m, float &v, const AdamConst &a) {
+__device__ __forceinline__ void adamw_elem(double g64, float &p, float &m, float &v, const AdamDev &a,
+                                           const AdamStep &st) {
     const double m64 = fma(a.b1, double(m), a.c1 * g64);
     const double v64 = fma(a.b2, double(v), (a.c2 * g64) * g64);
     double root = 0.0;
@@ -645,10 +760,10 @@ __device__ __forceinline__ void adamw_elem(double g64, float &p, float &m, float
         const double r = v64 * y;
         root = fma(fma(-r, r, v64), 0.5 * y, r);         // r + (v - r^2) / (2 sqrt(v))
     }
-    const double denom = fma(root, a.inv_sqrt_bc2, a.eps);
+    const double denom = fma(root, st.inv_sqrt_bc2, a.eps);
     const double q = rcp_approx64(denom);
     const double inv = q * fma(-denom, q, 2.0);          // q (2 - denom q)
-    const double delta = fma(a.lr_wd, double(p), a.step_size * (m64 * inv));
+    const double delta = fma(a.lr_wd, double(p), st.step_size * (m64 * inv));
     p = __double2float_rn(double(p) - delta);
     m = __double2float_rn(m64);
     v = __double2float_rn(v64);
@@ -656,7 +771,7 @@ __device__ __forceinline__ void adamw_elem(double g64, float &p, float &m, float
 
 template <typename GT, int GOP, bool STORE_D>
 __device__ __forceinline__ void adamw_chunk(const Chunk &ch, const OptChunk &oc, float k, double beta,
-                                            double s, const AdamConst &a) {
+                                            double s, const AdamDev &a, const AdamStep &st) {
     const void *g = reinterpret_cast<const void *>(ch.g);
     void *d = reinterpret_cast<void *>(ch.d);
     void *pp = reinterpret_cast<void *>(oc.p);
@@ -668,33 +783,38 @@ __device__ __forceinline__ void adamw_chunk(const Chunk &ch, const OptChunk &oc,
     if (vec) {
         const uint32_t nvec = ch.n >> 2;
         for (uint32_t base = 0; base < nvec; base += T * U) {
-            F4 gv[U], dv[U], p4[U], m4[U], v4[U];
+            typename Elem<GOf<GT>>::Raw gr[U];
+            typename Elem<DOf<GT>>::Raw dr[U];
+            float4 p4[U], m4[U], v4[U];
 #pragma unroll
             for (int u = 0; u < U; ++u) {
                 const uint32_t w = base + u * T + tid;
-                dv[u] = F4{0.f, 0.f, 0.f, 0.f};
+                gr[u] = Elem<GOf<GT>>::zero();
+                dr[u] = Elem<DOf<GT>>::zero();
+                p4[u] = m4[u] = v4[u] = make_float4(0.f, 0.f, 0.f, 0.f);
                 if (w < nvec) {
-                    gv[u] = Elem<GOf<GT>>::template load4<GAC_LD_PROJECT>(g, w);
-                    if (GOP == G_FMA) dv[u] = Elem<DOf<GT>>::template load4<GAC_LD_PROJECT>(d, w);
-                    p4[u] = Elem<float>::load4<GAC_LD_PROJECT>(pp, w);
-                    m4[u] = Elem<float>::load4<GAC_LD_PROJECT>(pm, w);
-                    v4[u] = Elem<float>::load4<GAC_LD_PROJECT>(pv, w);
+                    gr[u] = Elem<GOf<GT>>::template load_raw<GAC_LD_PROJECT>(g, w);
+                    if (GOP == G_FMA || GOP == G_FMA1) dr[u] = Elem<DOf<GT>>::template load_raw<GAC_LD_PROJECT>(d, w);
+                    p4[u] = Elem<float>::load_raw<GAC_LD_PROJECT>(pp, w);
+                    m4[u] = Elem<float>::load_raw<GAC_LD_PROJECT>(pm, w);
+                    v4[u] = Elem<float>::load_raw<GAC_LD_PROJECT>(pv, w);
                 }
             }
 #pragma unroll
             for (int u = 0; u < U; ++u) {
                 const uint32_t w = base + u * T + tid;
                 if (w >= nvec) continue;
-                float ge[4] = {gv[u].x, gv[u].y, gv[u].z, gv[u].w};
+                const F4 gq = Elem<GOf<GT>>::unpack(gr[u]), dq = Elem<DOf<GT>>::unpack(dr[u]);
+                const float ge[4] = {gq.x, gq.y, gq.z, gq.w};
                 float pe[4] = {p4[u].x, p4[u].y, p4[u].z, p4[u].w};
                 float me[4] = {m4[u].x, m4[u].y, m4[u].z, m4[u].w};
                 float ve[4] = {v4[u].x, v4[u].y, v4[u].z, v4[u].w};
-                const float de[4] = {dv[u].x, dv[u].y, dv[u].z, dv[u].w};
+                const float de[4] = {dq.x, dq.y, dq.z, dq.w};
 #pragma unroll
                 for (int e = 0; e < 4; ++e) {
-                    adamw_elem(outgoing64<GOP>(ge[e], de[e], k, beta, s), pe[e], me[e], ve[e], a);
+                    adamw_elem(outgoing64<GOP>(ge[e], de[e], k, beta, s), pe[e], me[e], ve[e], a, st);
                 }
-                if (STORE_D) Elem<DOf<GT>>::store4(d, w, gv[u]);          // d' = g, the raw gradient
+                if (STORE_D) Elem<DOf<GT>>::store4(d, w, gq);             // d' = g, the raw gradient
                 Elem<float>::store4(pp, w, F4{pe[0], pe[1], pe[2], pe[3]});
                 Elem<float>::store4(pm, w, F4{me[0], me[1], me[2], me[3]});
                 Elem<float>::store4(pv, w, F4{ve[0], ve[1], ve[2], ve[3]});
@@ -704,9 +824,9 @@ __device__ __forceinline__ void adamw_chunk(const Chunk &ch, const OptChunk &oc,
     const uint32_t first = vec ? ((ch.n >> 2) << 2) : 0u;
     for (uint32_t i = first + tid; i < ch.n; i += T) {
         const float x = Elem<GOf<GT>>::load1(g, i);
-        const float dx = (GOP == G_FMA) ? Elem<DOf<GT>>::load1(d, i) : 0.f;
+        const float dx = (GOP == G_FMA || GOP == G_FMA1) ? Elem<DOf<GT>>::load1(d, i) : 0.f;
         float pe = Elem<float>::load1(pp, i), me = Elem<float>::load1(pm, i), ve = Elem<float>::load1(pv, i);
-        adamw_elem(outgoing64<GOP>(x, dx, k, beta, s), pe, me, ve, a);
+        adamw_elem(outgoing64<GOP>(x, dx, k, beta, s), pe, me, ve, a, st);
         if (STORE_D) Elem<DOf<GT>>::store1(d, i, x);
         Elem<float>::store1(pp, i, pe);
         Elem<float>::store1(pm, i, me);
@@ -737,10 +857,9 @@ __global__ void __launch_bounds__(AdamGeom<GT>::T, AdamGeom<GT>::C)
 gac_adamw_kernel(const Chunk *__restrict__ chunks, const OptChunk *__restrict__ opt_chunks,
                  uint32_t n_chunks, gac_result *rec, unsigned *ticket, float coef_override,
                  int use_override, double beta, double clip_max, double clip_eps, AdamDev o, int swapped) {
-    if (rec->nonfinite) {
-        if (EXCH && blockIdx.x == 0 && threadIdx.x == 0) rec->ref_lost = 1u;
-        return;
-    }
+    const bool closed = rec->nonfinite || rec->timed_out;
+    if (EXCH && blockIdx.x == 0 && threadIdx.x == 0) rec->ref_lost = closed ? 1u : 0u;
+    if (closed) return;
     const int regime = rec->regime;
     const float k = use_override ? coef_override : rec->coef;
     const unsigned long long t_prev = rec->applied_steps;
@@ -756,22 +875,20 @@ gac_adamw_kernel(const Chunk *__restrict__ chunks, const OptChunk *__restrict__ 
     const bool applies = (regime != GAC_REGIME_VIOLATION);
     if (applies) {
         const double t = double(t_prev + 1ull);
-        const double bc1 = 1.0 - pow(o.beta1, t), bc2 = 1.0 - pow(o.beta2, t);
-        AdamConst a;
-        a.b1 = o.beta1;
-        a.c1 = 1.0 - o.beta1;
-        a.b2 = o.beta2;
-        a.c2 = 1.0 - o.beta2;
-        a.step_size = o.lr / bc1;
-        a.inv_sqrt_bc2 = 1.0 / sqrt(bc2);
-        a.eps = o.eps;
-        a.lr_wd = o.lr * o.weight_decay;
+        const double bc1 = 1.0 - pow(o.b1, t), bc2 = 1.0 - pow(o.b2, t);
+        AdamStep st;
+        st.step_size = o.lr / bc1;
+        st.inv_sqrt_bc2 = 1.0 / sqrt(bc2);
+        // one uniform choice per launch; each branch holds only the loop it needs
+        const int gop = regime == GAC_REGIME_PROJECT ? ((beta == 1.0 && s == 1.0) ? G_FMA1 : G_FMA)
+                                                     : (s != 1.0 ? G_SCALE : G_KEEP);
         for (uint32_t c = blockIdx.x; c < n_chunks; c += gridDim.x) {
             const Chunk ch = load_chunk(chunks, c, swapped);
             const OptChunk oc = load_opt_chunk(opt_chunks, c);
-            if (regime == GAC_REGIME_PROJECT) adamw_chunk<GT, G_FMA, !EXCH>(ch, oc, k, beta, s, a);
-            else if (s != 1.0) adamw_chunk<GT, G_SCALE, !EXCH>(ch, oc, k, 1.0, s, a);
-            else adamw_chunk<GT, G_KEEP, !EXCH>(ch, oc, k, 1.0, 1.0, a);
+            if (gop == G_FMA1) adamw_chunk<GT, G_FMA1, !EXCH>(ch, oc, k, 1.0, 1.0, o, st);
+            else if (gop == G_FMA) adamw_chunk<GT, G_FMA, !EXCH>(ch, oc, k, beta, s, o, st);
+            else if (gop == G_SCALE) adamw_chunk<GT, G_SCALE, !EXCH>(ch, oc, k, 1.0, s, o, st);
+            else adamw_chunk<GT, G_KEEP, !EXCH>(ch, oc, k, 1.0, 1.0, o, st);
         }
     } else if (!EXCH) {
         for (uint32_t c = blockIdx.x; c < n_chunks; c += gridDim.x)   // skipped step: d' = g only
@@ -782,7 +899,8 @@ gac_adamw_kernel(const Chunk *__restrict__ chunks, const OptChunk *__restrict__ 
         __threadfence();
         const unsigned done = atomicAdd(ticket, 1u);
         if (done == gridDim.x - 1) {
-            rec->applied_steps = t_prev + (applies ? 1ull : 0ull);
+            // read again rather than held across the loop: nobody has written it during this launch
+            rec->applied_steps = rec->applied_steps + (rec->regime != GAC_REGIME_VIOLATION ? 1ull : 0ull);
             __threadfence();
             *ticket = 0u;
         }

@@ -49,14 +49,51 @@ def shard_views(tensors: Sequence[torch.Tensor], pieces: Sequence[Piece]) -> Lis
 
 
 def sharded_step(gb, ctx, step: int, sums: torch.Tensor, group=None, staleness: int = 0,
-                 fetch: bool = False, coef_override=None):
+                 fetch: bool = False, coef_override=None, mark=None, peer_exchange: bool = False):
     """One GAC step on this rank's shard: local sums -> all-reduce of three
     doubles -> decision -> in-place update.  `gb` is the binding module, `sums`
     a float64 CUDA tensor of 3 elements reused across steps.  All calls are
-    enqueued on the current stream; the collective is NCCL's."""
-    gb.gac_stats_partial(ctx, step, sums, staleness=staleness)
-    if dist.is_available() and dist.is_initialized() and dist.get_world_size(group) > 1:
-        dist.all_reduce(sums, op=dist.ReduceOp.SUM, group=group)
-    res = gb.gac_decide(ctx, sums, fetch=fetch)
+    enqueued on the current stream; the collective is the process group's
+    (NCCL on GPUs) -- or, with `peer_exchange` on a context prepared by
+    `attach_peer_exchange`, the library's own: the reduction kernel stores the
+    three sums into every rank's slot array and a small kernel adds them in
+    rank order.  `mark`, if given, is called once the decision has been
+    enqueued and before the update is (a caller that times the two passes
+    records an event there).  Returns the decision record when `fetch`."""
+    if peer_exchange:
+        gb.gac_stats_exchange(ctx, step, staleness=staleness)
+        res = gb.gac_decide_exchange(ctx, fetch=fetch)
+    else:
+        gb.gac_stats_partial(ctx, step, sums, staleness=staleness)
+        if dist.is_available() and dist.is_initialized():
+            dist.all_reduce(sums, op=dist.ReduceOp.SUM, group=group)
+        res = gb.gac_decide(ctx, sums, fetch=fetch)
+    if mark is not None:
+        mark()
     gb.gac_project(ctx, coef_override=coef_override)
     return res
+
+
+def attach_peer_exchange(gb, ctx, group=None, timeout_ms: int = 0):
+    """Prepares a context for `sharded_step(..., peer_exchange=True)`: allocates this rank's slot
+    array in symmetric memory, lets every rank map every other rank's array (a collective over
+    `group`; PyTorch's symmetric memory does the mapping), zero-fills it and hands the addresses
+    to the library.  Returns the symmetric-memory tensor, which the caller must keep alive as long
+    as the context is used.  Raises if symmetric memory cannot be set up; NCCL's all-reduce (the
+    default path of `sharded_step`) needs none of this."""
+    import torch.distributed._symmetric_memory as symm
+    if not (dist.is_available() and dist.is_initialized()):
+        raise RuntimeError("attach_peer_exchange needs an initialised process group")
+    pg = group if group is not None else dist.group.WORLD
+    world, rank = dist.get_world_size(pg), dist.get_rank(pg)
+    buf = symm.empty(gb.gac_exchange_bytes(world), dtype=torch.uint8, device=torch.device("cuda", torch.cuda.current_device()))
+    handle = symm.rendezvous(buf, pg)
+    buf.zero_()
+    torch.cuda.synchronize()
+    dist.barrier(group=pg)                 # nobody posts before every array reads zero
+    slots = [int(p) for p in handle.buffer_ptrs]
+    if len(slots) != world or slots[rank] != buf.data_ptr():
+        raise RuntimeError("symmetric memory returned an unexpected set of buffer addresses")
+    gb.gac_exchange_attach(ctx, rank, world, slots, timeout_ms)
+    ctx._keep_symm = (buf, handle)
+    return buf

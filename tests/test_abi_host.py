@@ -113,6 +113,26 @@ def test_argument_errors_need_no_device(lib):
         assert rc == gb.GAC_ERR_CUDA and "device" in msg
 
 
+def test_static_entry_argument_errors_need_no_device(lib):
+    """gac_stats_static checks its arguments before it touches CUDA: a misaligned record pointer (the
+    record holds doubles, a 4-byte aligned address would make the device stores fault) is refused on
+    the host, with a message."""
+    hp = gb.gac_hparams()
+    lib.gac_default_hparams(ctypes.byref(hp))
+    arr = (gb.gac_tensor * 1)(gb.gac_tensor(4096, 8192, 16))
+
+    def call(result_ptr, step=2, n=1, g_dt=0, d_dt=0):
+        rc = lib.gac_stats_static(arr, n, g_dt, d_dt, ctypes.byref(hp), step, 0, 0, None, result_ptr)
+        return rc, lib.gac_last_error(None).decode()
+
+    rc, msg = call(0x10004)
+    assert rc == gb.GAC_ERR_INVALID_ARG and "8-byte aligned" in msg
+    assert call(None)[0] == gb.GAC_ERR_INVALID_ARG
+    assert call(0x10000, step=0)[0] == gb.GAC_ERR_INVALID_ARG
+    assert call(0x10000, n=0)[0] == gb.GAC_ERR_INVALID_ARG
+    assert call(0x10000, g_dt=0, d_dt=1)[0] == gb.GAC_ERR_DTYPE
+
+
 def test_null_context_is_rejected(lib):
     r = gb.gac_result()
     assert lib.gac_stats(None, 1, 0, None, ctypes.byref(r)) == gb.GAC_ERR_INVALID_ARG

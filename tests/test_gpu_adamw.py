@@ -114,3 +114,84 @@ def test_fused_adamw_larger_list_and_call_rules():
         gb.gac_attach_adamw(ctx, z, z, z)
     assert e.value.status == gb.GAC_ERR_INVALID_ARG
     gb.gac_free(ctx)
+
+
+def ulp32(x: torch.Tensor) -> torch.Tensor:
+    """Spacing of binary32 numbers at magnitude x (float64 tensor)."""
+    e = torch.floor(torch.log2(x.abs().clamp_min(2.0 ** -126)))
+    return torch.pow(torch.tensor(2.0, dtype=torch.float64), e - 23)
+
+
+@pytest.mark.parametrize("opt_kw", [dict(), dict(lr=1e-3, weight_decay=0.1)], ids=["table2", "large_lr"])
+@pytest.mark.parametrize("g_dtype", [torch.float32, torch.bfloat16], ids=["f32", "bf16"])
+def test_fused_adamw_free_running_trajectory(g_dtype, opt_kw):
+    """p, m and v are carried on the GPU for 8 steps and never reset to the oracle's values.  Both sides
+    round m, v and p once per step, so per step they can part by one binary32 spacing of the new value;
+    an earlier difference is carried on times b1 (m), b2 (v), 1 (p), and reaches p through the update
+    lr_t m / (sqrt(v)/sqrt(1-b2^t) + eps) to first order.  The bound below is exactly that recurrence,
+    evaluated on the oracle's values (plus the binary64 noise terms the per-step test uses)."""
+    shapes = synth.decoder_tensor_list(synth.DIMS["mini"])
+    sig = synth.per_tensor_scales(2, len(shapes))
+    gen = torch.Generator().manual_seed(21)
+    hp = gb.HParams()
+    ohp = to_orc_hp(hp)
+    gopt, oopt = gb.AdamW(**opt_kw), orc.AdamW(**opt_kw)
+    p_cpu = [torch.randn(n, generator=gen) * 0.02 for _, n in shapes]
+    m_cpu = [torch.zeros(n) for _, n in shapes]
+    v_cpu = [torch.zeros(n) for _, n in shapes]
+    d_cpu = [torch.full((n,), float("nan")) for _, n in shapes]
+    g_gpu = [torch.empty(n, dtype=g_dtype, device="cuda") for _, n in shapes]
+    d_gpu = [t.cuda() for t in d_cpu]
+    p_gpu, m_gpu, v_gpu = ([t.cuda() for t in l] for l in (p_cpu, m_cpu, v_cpu))
+    ctx = gb.gac_init(g_gpu, d_gpu, hp)
+    gb.gac_attach_adamw(ctx, p_gpu, m_gpu, v_gpu, applied_steps=0)
+    err_m = [torch.zeros(n, dtype=torch.float64) for _, n in shapes]
+    err_v = [torch.zeros(n, dtype=torch.float64) for _, n in shapes]
+    err_p = [torch.zeros(n, dtype=torch.float64) for _, n in shapes]
+    prev = [torch.randn(n, generator=gen) * s for (_, n), s in zip(shapes, sig)]
+    applied, regimes = 0, []
+    for t, rho in enumerate((None, 0.0, 0.15, 0.9, 0.2, 0.01, 0.25, 0.1), start=1):
+        noise = [torch.randn(n, generator=gen) * s for (_, n), s in zip(shapes, sig)]
+        g = noise if rho is None else [rho * a + math.sqrt(1 - rho * rho) * b for a, b in zip(prev, noise)]
+        g = [x.to(g_dtype) for x in g]
+        prev = [x.float() for x in g]
+        for dst, src in zip(g_gpu, g):
+            dst.copy_(src)
+        first = t == 1
+        dec = orc.decide(orc.stats(g, d_cpu, first_step=first), ohp, first)
+        m_before = [x.double() for x in m_cpu]
+        v_before = [x.double() for x in v_cpu]
+        gmag = [x.double().abs() + abs(dec.coef) * y.double().abs().nan_to_num(0.0) for x, y in zip(g, d_cpu)]
+        did = orc.project_adamw(g, d_cpu, p_cpu, m_cpu, v_cpu, ohp, dec, oopt, applied + 1, first)
+        applied += int(did)
+        gb.gac_stats(ctx, t, fetch=False)
+        after = gb.gac_project_adamw(ctx, gopt, coef_override=dec.coef if dec.regime == orc.PROJECT else None,
+                                     fetch=True)
+        assert after.regime == dec.regime and after.applied_steps == applied
+        regimes.append(dec.regime)
+        if did:
+            step_size = oopt.lr / (1.0 - oopt.beta1 ** applied)
+            isb2 = 1.0 / math.sqrt(1.0 - oopt.beta2 ** applied)
+            for i in range(len(shapes)):
+                m_new, v_new = m_cpu[i].double(), v_cpu[i].double()
+                err_m[i] = oopt.beta1 * err_m[i] + ulp32(m_new) + 1e-13 * (m_before[i].abs() + gmag[i])
+                err_v[i] = oopt.beta2 * err_v[i] + ulp32(v_new) + 1e-13 * (v_before[i] + gmag[i] ** 2)
+                root = v_new.sqrt()
+                denom = root * isb2 + oopt.eps
+                d_denom = isb2 * err_v[i] / (root + 1e-300)
+                d_update = step_size * (err_m[i] / denom + m_new.abs() * d_denom / denom ** 2)
+                err_p[i] = err_p[i] + ulp32(p_cpu[i].double()) + d_update + 1e-10 * oopt.lr
+        for i in range(len(shapes)):
+            assert torch.equal(d_gpu[i].cpu(), d_cpu[i]), "stored direction is not the raw gradient"
+            for name, a, b, err in (("m", m_gpu[i], m_cpu[i], err_m[i]), ("v", v_gpu[i], v_cpu[i], err_v[i]),
+                                    ("p", p_gpu[i], p_cpu[i], err_p[i])):
+                diff = (a.cpu().double() - b.double()).abs()
+                bad = diff > err
+                assert not bool(bad.any()), (f"step {t} tensor {i} {name}: off by {float(diff[bad].max()):.3e}, "
+                                             f"bound {float(err[bad].min()):.3e}")
+    gb.gac_free(ctx)
+    assert set(regimes) == {orc.SAFE, orc.PROJECT, orc.VIOLATION} and applied >= 5
+    # the bound stays a rounding-level statement: a few binary32 spacings of p per step, plus a
+    # 1e-5-th of one update where p itself is tiny
+    for i in range(len(shapes)):
+        assert bool((err_p[i] <= 8 * 4 * ulp32(p_cpu[i].double()) + 1e-5 * oopt.lr).all())

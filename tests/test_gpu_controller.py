@@ -97,3 +97,65 @@ def test_controller_in_exchange_mode_matches_the_raw_rule():
     with pytest.raises(RuntimeError):
         ctl.step()
     ctl.close()
+
+
+@pytest.mark.parametrize("exchange", [False, True], ids=["copy", "exchange"])
+def test_controller_resumes_from_its_state_dict(exchange):
+    """Save after step 3, build a new controller, load, go on: steps 4 and 5 must equal those of the
+    uninterrupted run bit for bit (sums, decision, outgoing gradient, stored direction)."""
+    gen = torch.Generator().manual_seed(5)
+    sizes = [1000, 33, 70001, 4096]
+    seq, prev = [], None
+    for rho in (None, 0.2, 0.7, 0.15, 0.3):       # safe first step, then projections and a violation
+        noise = [torch.randn(n, generator=gen) for n in sizes]
+        g = noise if prev is None else [rho * a + (1 - rho * rho) ** 0.5 * b for a, b in zip(prev, noise)]
+        seq.append(g)
+        prev = g
+    hp = gb.HParams(c_low=0.05, c_high=0.6)
+
+    def feed(ctl, params, g, first):
+        if exchange and not first:
+            ctl.zero_grad()
+            for p, x in zip(params, g):
+                p.grad.copy_(x.view_as(p))
+        else:
+            for p, x in zip(params, g):
+                p.grad = x.clone().cuda().view_as(p)
+
+    def snap(ctl, params, take):
+        r = ctl.last
+        return (take, r.dot, r.gg, r.dd, r.cos, r.coef, r.regime, r.step,
+                [p.grad.detach().view(-1).cpu().clone() for p in params],
+                [s.cpu().clone() for s in ctl.snapshot])
+
+    def same(a, b):
+        assert a[:8] == b[:8]
+        for x, y in zip(a[8] + a[9], b[8] + b[9]):
+            assert torch.equal(x.view(torch.int32), y.view(torch.int32))
+
+    params = [torch.nn.Parameter(torch.zeros(n, device="cuda")) for n in sizes]
+    ctl = GradientAlignmentController(params, hp, exchange=exchange)
+    whole = []
+    for t, g in enumerate(seq):
+        feed(ctl, params, g, t == 0)
+        whole.append(snap(ctl, params, ctl.step()))
+    ctl.close()
+    assert {w[6] for w in whole} == {orc.SAFE, orc.PROJECT, orc.VIOLATION}
+
+    params = [torch.nn.Parameter(torch.zeros(n, device="cuda")) for n in sizes]
+    ctl = GradientAlignmentController(params, hp, exchange=exchange)
+    for t, g in enumerate(seq[:3]):
+        feed(ctl, params, g, t == 0)
+        same(snap(ctl, params, ctl.step()), whole[t])
+    state = ctl.state_dict()
+    ctl.close()
+    assert state["t"] == 3
+
+    params = [torch.nn.Parameter(torch.zeros(n, device="cuda")) for n in sizes]
+    ctl = GradientAlignmentController(params, hp, exchange=exchange)
+    feed(ctl, params, seq[3], True)               # the gradient of step 4 exists before the state is loaded
+    ctl.load_state_dict(state)
+    same(snap(ctl, params, ctl.step()), whole[3])
+    feed(ctl, params, seq[4], False)
+    same(snap(ctl, params, ctl.step()), whole[4])
+    ctl.close()

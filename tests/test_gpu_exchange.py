@@ -130,6 +130,39 @@ def test_exchange_mode_restarts_after_a_nonfinite_step(dtype):
     assert regimes[2] == "nonfinite" and regimes[3] == orc.SAFE and regimes[4] == orc.PROJECT
 
 
+def test_exchange_mode_statistics_pass_is_idempotent_after_a_nonfinite_step():
+    """The reduction may run more than once for a step.  After a non-finite step the stored direction
+    is lost; every reduction of the following step must then take the zero reference -- the mark
+    stays until the pass that closes that step clears it."""
+    n = 50000
+    a = torch.randn(n, device="cuda")
+    b = torch.randn(n, device="cuda")
+    ctx = gb.gac_init([a], [b], gb.HParams(state_mode=gb.GAC_STATE_EXCHANGE))
+    gb.gac_stats(ctx, 1)
+    gb.gac_project(ctx)                       # a holds the stored direction, b takes the next gradient
+    b.copy_(torch.randn(n, device="cuda"))
+    b[17] = float("inf")
+    r = gb.gac_stats(ctx, 2)
+    after = gb.gac_project(ctx, fetch=True)
+    assert r.nonfinite == 1 and after.ref_lost == 1
+    a.copy_(torch.randn(n, device="cuda"))    # step 3: gradient in a; b still holds the Inf
+    gg = float((a.double() ** 2).sum())
+    first = gb.gac_stats(ctx, 3)
+    second = gb.gac_stats(ctx, 3)
+    third = gb.gac_stats(ctx, 3)
+    for r in (first, second, third):
+        assert (r.nonfinite, r.regime, r.dot, r.dd, r.cos) == (0, gb.GAC_REGIME_SAFE, 0.0, 0.0, 0.0)
+        assert r.gg == first.gg and abs(r.gg - gg) <= 1e-9 * gg and r.ref_lost == 1
+    after = gb.gac_project(ctx, fetch=True)
+    assert after.ref_lost == 0
+    # step 4 compares against step 3's gradient again
+    b.copy_(0.5 * a + 0.1 * torch.randn(n, device="cuda"))
+    r = gb.gac_stats(ctx, 4)
+    assert r.nonfinite == 0 and r.dd == first.gg and abs(r.cos) > 0.9
+    gb.gac_project(ctx)
+    gb.gac_free(ctx)
+
+
 @pytest.mark.parametrize("hp", [
     gb.HParams(state_mode=gb.GAC_STATE_EXCHANGE, zero_on_violation=1),
     gb.HParams(state_mode=gb.GAC_STATE_EXCHANGE, clip_max_norm=1e-3),

@@ -341,6 +341,21 @@ def test_call_order_is_enforced():
     gb.gac_stats(ctx, 6)
     info = gb.gac_get_info(ctx)
     assert info.launches == 3 and info.total_elems == 100
+    # three doubles at a 4-byte aligned address would make the device stores fault: refused on the
+    # host, nothing is launched
+    import ctypes
+    lib = gb.load_library()
+    odd = torch.zeros(8, dtype=torch.float32, device="cuda")
+    assert (odd.data_ptr() + 4) % 8 == 4
+    rc = lib.gac_stats_partial(ctx.handle, 7, 0, None, ctypes.c_void_p(odd.data_ptr() + 4))
+    assert rc == gb.GAC_ERR_INVALID_ARG and b"8-byte aligned" in lib.gac_last_error(ctx.handle)
+    sums = torch.zeros(3, dtype=torch.float64, device="cuda")
+    gb.gac_stats_partial(ctx, 7, sums)
+    rc = lib.gac_decide(ctx.handle, None, ctypes.c_void_p(odd.data_ptr() + 4), None)
+    assert rc == gb.GAC_ERR_INVALID_ARG and b"8-byte aligned" in lib.gac_last_error(ctx.handle)
+    gb.gac_decide(ctx, sums)
+    gb.gac_project(ctx)
+    assert gb.gac_get_info(ctx).launches == 6
     gb.gac_free(ctx)
 
 

@@ -12,6 +12,7 @@ import ctypes
 import pytest
 import torch
 
+from oracle import gac_oracle as orc
 from paper_2603_01501_b200 import binding as gb
 from paper_2603_01501_b200 import synth
 
@@ -76,3 +77,58 @@ def test_static_scratch_first_step_and_limits():
     assert e.value.status == gb.GAC_ERR_INVALID_ARG and "scratch" in str(e.value)
     with pytest.raises(gb.GacError):
         gb.gac_stats_static(g, d, hp, 0, out)
+
+
+def test_static_scratch_against_the_oracle_and_free_memory_unchanged():
+    """The property the entry point exists for: ten calls in a row leave the amount of free device
+    memory exactly where it was.  The float32 result is checked against the CPU oracle as well, and
+    the fields the reduction does not own come back as zero although the record was pre-filled."""
+    hp = gb.HParams(c_low=0.05, c_high=2.0)
+    shapes = synth.decoder_tensor_list(synth.DIMS["small"])
+    g_cpu, d_cpu = synth.gradient_list(shapes, 0.7, config_id=2)
+    dec = orc.decide(orc.stats(g_cpu, d_cpu), orc.HParams(c_low=0.05, c_high=2.0))
+    g = [t.cuda() for t in g_cpu]
+    d = [t.cuda() for t in d_cpu]
+    out = torch.zeros(ctypes.sizeof(gb.gac_result), dtype=torch.uint8, device="cuda")
+    gb.gac_stats_static(g, d, hp, 2, out)          # the first call on a device looks up the array's address
+    torch.cuda.synchronize()
+    free_before, _ = torch.cuda.mem_get_info()
+    for step in range(2, 12):
+        out.fill_(0xAB)
+        gb.gac_stats_static(g, d, hp, step, out)
+    torch.cuda.synchronize()
+    free_after, _ = torch.cuda.mem_get_info()
+    assert free_after == free_before
+    got = gb.result_from_tensor(out)
+    scale = 1e-6 * (dec.gg * dec.dd) ** 0.5
+    assert _close(got.gg, dec.gg) and _close(got.dd, dec.dd) and _close(got.dot, dec.dot, scale)
+    assert _close(got.cos, dec.cos, 1e-6) and got.regime == dec.regime == orc.PROJECT
+    assert _close(got.alpha, dec.alpha) and _close(got.coef, dec.coef)
+    assert (got.step, got.applied_steps, got.ref_lost, got.g_set, got.out_set) == (11, 0, 0, 0, 0)
+
+
+def test_static_scratch_is_refused_on_a_capturing_stream():
+    """A captured call would replay its table copy from the library's shared host buffer as it stands
+    at replay time: the entry point refuses instead, enqueues nothing, and the capture stays valid."""
+    hp = gb.HParams()
+    g = [torch.randn(70000, device="cuda")]
+    d = [torch.randn(70000, device="cuda")]
+    out = torch.zeros(ctypes.sizeof(gb.gac_result), dtype=torch.uint8, device="cuda")
+    gb.gac_stats_static(g, d, hp, 2, out)          # set-up happens outside the capture
+    torch.cuda.synchronize()
+    want = gb.result_from_tensor(out)
+    side = torch.cuda.Stream()
+    graph = torch.cuda.CUDAGraph()
+    marker = torch.zeros(4, device="cuda")
+    with torch.cuda.stream(side):
+        graph.capture_begin()
+        with pytest.raises(gb.GacError) as e:
+            gb.gac_stats_static(g, d, hp, 3, out, stream=side)
+        marker.add_(1.0)                            # the capture goes on: the refusal broke nothing
+        graph.capture_end()
+    assert e.value.status == gb.GAC_ERR_STATE and "captured" in str(e.value)
+    graph.replay()
+    torch.cuda.synchronize()
+    assert marker.tolist() == [1.0] * 4
+    again = gb.result_from_tensor(out)
+    assert (again.step, again.gg, again.dot) == (want.step, want.gg, want.dot)     # untouched by the refused call
