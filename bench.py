@@ -236,6 +236,7 @@ class Workload:
 
     def close(self):
         self.gb.gac_free(self.ctx)
+        self.ctx = None
         self.g = self.d = self.scratch = None
         torch.cuda.empty_cache()
 

@@ -14,7 +14,9 @@ from typing import List, Optional, Sequence
 import torch
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_HERE, "libgac_b200.so")
+# GAC_B200_LIBRARY selects another build of the same library (a debug build, or one compiled with
+# another launch-geometry table through -DGAC_GEOMETRY_HEADER); the default is the in-tree build.
+LIB_PATH = os.environ.get("GAC_B200_LIBRARY") or os.path.join(_HERE, "libgac_b200.so")
 
 GAC_OK, GAC_ERR_INVALID_ARG, GAC_ERR_DTYPE, GAC_ERR_CUDA, GAC_ERR_STATE, GAC_ERR_NONFINITE, \
     GAC_ERR_TIMEOUT = range(7)
@@ -307,6 +309,11 @@ def gac_free(ctx: GacContext) -> None:
     if ctx.handle:
         load_library().gac_free(ctx.handle)
         ctx.handle = ctypes.c_void_p(None)
+    # the library no longer touches the buffers: let go of them, so that their owner can free them
+    ctx._keep = ([], [])
+    for extra in ("_keep_opt", "_keep_slots", "_keep_symm"):
+        if hasattr(ctx, extra):
+            setattr(ctx, extra, None)
 
 
 def gac_set_launch(ctx: GacContext, chunk_elems: int = 0, ctas_per_sm: int = 0) -> None:

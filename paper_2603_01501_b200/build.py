@@ -31,5 +31,25 @@ def build(force: bool = False, verbose: bool = False) -> str:
     return LIB
 
 
+PROBE_SRC = os.path.join(HERE, "csrc", "stream_probe.cu")
+PROBE = os.path.join(HERE, "stream_probe")
+
+
+def build_probe(force: bool = False) -> str:
+    """Builds the stand-alone HBM stream-pattern probe (an executable, not part of the library)."""
+    if not force and os.path.exists(PROBE) and os.path.getmtime(PROBE) >= os.path.getmtime(PROBE_SRC):
+        return PROBE
+    nvcc = os.environ.get("NVCC", "nvcc")
+    cmd = [nvcc, "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17", "-o", PROBE, PROBE_SRC]
+    proc = subprocess.run(cmd, capture_output=True, text=True)
+    if proc.returncode != 0:
+        sys.stderr.write(proc.stdout + proc.stderr)
+        raise RuntimeError("nvcc failed: " + " ".join(cmd))
+    return PROBE
+
+
 if __name__ == "__main__":
-    print(build(force=True, verbose=True))
+    if len(sys.argv) > 1 and sys.argv[1] == "probe":
+        print(build_probe(force=True))
+    else:
+        print(build(force=True, verbose=True))
