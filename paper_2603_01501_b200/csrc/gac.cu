@@ -204,7 +204,10 @@ int build_opt_table(gac_ctx *c) {
     GAC_CUDA(c, cudaMalloc(&c->d_opt_chunks, table.size() * sizeof(OptChunk)));
     GAC_CUDA(c, cudaMemcpy(c->d_opt_chunks, table.data(), table.size() * sizeof(OptChunk),
                            cudaMemcpyHostToDevice));
-    c->threads_adamw = with_pair(c->pair, [](auto tag) { return AdamGeom<decltype(tag)>::T; });
+    const bool plain = (c->hp.beta == 1.0 && c->hp.clip_max_norm == 0.0);   // the paper's own rule: the leaner instantiation
+    c->threads_adamw = with_pair(c->pair, [plain](auto tag) {
+        return plain ? AdamGeom<decltype(tag)>::T : AdamGeom<decltype(tag)>::TG;
+    });
     const int ctas = with_pair(c->pair, [](auto tag) { return AdamGeom<decltype(tag)>::C; });
     c->grid_adamw = int(std::min<uint64_t>(uint64_t(c->sms) * ctas, c->n_chunks));
     return GAC_OK;
@@ -671,8 +674,11 @@ int gac_project_adamw(gac_ctx *ctx, void *cuda_stream, const gac_adamw *opt, con
     const AdamDev o{opt->lr, opt->beta1, opt->beta2, opt->eps, 1.0 - opt->beta1, 1.0 - opt->beta2,
                     opt->lr * opt->weight_decay};
     const bool exch = (ctx->hp.state_mode == GAC_STATE_EXCHANGE);
-    const AdamKernel ak = with_pair(ctx->pair, [exch](auto tag) -> AdamKernel {
-        return exch ? gac_adamw_kernel<decltype(tag), true> : gac_adamw_kernel<decltype(tag), false>;
+    const bool plain = (ctx->hp.beta == 1.0 && ctx->hp.clip_max_norm == 0.0);
+    const AdamKernel ak = with_pair(ctx->pair, [exch, plain](auto tag) -> AdamKernel {
+        using P = decltype(tag);
+        if (plain) return exch ? gac_adamw_kernel<P, true, true> : gac_adamw_kernel<P, false, true>;
+        return exch ? gac_adamw_kernel<P, true, false> : gac_adamw_kernel<P, false, false>;
     });
     ak<<<ctx->grid_adamw, ctx->threads_adamw, 0, s>>>(ctx->d_chunks, ctx->d_opt_chunks, nc, ctx->d_rec, ctx->d_ticket,
                                                       k, use, ctx->hp.beta, ctx->hp.clip_max_norm, ctx->hp.clip_eps, o,

@@ -1,20 +1,27 @@
 // stream_probe -- what HBM delivers for the access patterns of this library's kernels, with the
 // arithmetic taken out: R read streams and W write streams of float4, each its own allocation,
 // cut into 64 KB chunks that the CTAs take round-robin (chunk c -> CTA c mod grid), T threads
-// with U vectors of every read stream in flight per thread, streaming stores.
+// with U vectors of every read stream in flight per thread, streaming stores.  "in place" means
+// that the W results overwrite the last W of the R streams read (as the kernels update g, d, p,
+// m, v where they lie); otherwise the results go to W further allocations.
 //
 // The figures it prints are the ceilings the kernels are measured against besides the plain
 // copy rate: a kernel that matches the probe of its own pattern is limited by how DRAM serves
 // that mix of streams, not by its instructions.
 //
-//   stream_probe [elements per stream, default 2^30]
+//   stream_probe [elements per stream, default 2^30] [stagger bytes, default 0]
 //
-// Patterns: 1+1 (copy), 2+0 (fused triple reduction), 2+2 (projection + state refresh),
+// With a stagger, stream i starts i x stagger bytes into its allocation (a multiple of 16), so
+// that the streams no longer share their low address bits: allocations of one size that come
+// from one allocator usually do.
+//
+// Patterns: 2+0 (fused triple reduction), 2+2 (projection + state refresh),
 // 2+1 (projection in exchange mode), 5+4 and 5+3 (projection fused with AdamW, with and
 // without the state copy).  One line per pattern and geometry:
-//   streams R=.. W=.. T=.. U=.. ctas/sm=.. elems=.. ms=.. GB/s=..
+//   streams stagger=.. R=.. W=.. place=in|out after=same|read pipelined=yes|no T=.. U=.. ctas/sm=.. elems=.. ms=.. GB/s=..
 #include <cuda_runtime.h>
 
+#include <cstdint>
 #include <cstdio>
 #include <cstdlib>
 
@@ -34,21 +41,44 @@ struct Streams {
     float4 *p[kMaxStreams];
 };
 
-template <int R, int W, int T, int U>
-__global__ void __launch_bounds__(T, 1) walk(Streams s, size_t n_chunks) {
+template <int R, int U, int T>
+__device__ __forceinline__ void load_batch(float4 (&v)[R][U], float4 *const (&p)[R], uint32_t base, uint32_t chunk_vec) {
+#pragma unroll
+    for (int u = 0; u < U; ++u) {
+        const uint32_t i = base + u * T + threadIdx.x;
+#pragma unroll
+        for (int r = 0; r < R; ++r) v[r][u] = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (i < chunk_vec) {
+#pragma unroll
+            for (int r = 0; r < R; ++r) v[r][u] = p[r][i];
+        }
+    }
+}
+
+// PIPE: the loads of the next batch are issued before the results of the current one are stored,
+// so that a thread always has reads in flight while it writes.
+template <int R, int W, int T, int U, bool INPLACE, bool PIPE>
+__global__ void __launch_bounds__(T, 1) walk(Streams s, size_t n_chunks, uint32_t chunk_vec) {
+    constexpr int kFirstOut = INPLACE ? R - W : R;
+    const uint32_t tid = threadIdx.x;
     for (size_t c = blockIdx.x; c < n_chunks; c += gridDim.x) {
-        const size_t off = c * size_t(kChunkVec);
-        for (int base = 0; base < kChunkVec; base += T * U) {
-            float4 v[R][U];
+        float4 *in[R], *out[W > 0 ? W : 1];   // the chunk's first vector in every stream
 #pragma unroll
-            for (int u = 0; u < U; ++u) {
-                const int i = base + u * T + threadIdx.x;
+        for (int i = 0; i < R; ++i) in[i] = s.p[i] + c * size_t(chunk_vec);
 #pragma unroll
-                for (int r = 0; r < R; ++r) v[r][u] = i < kChunkVec ? s.p[r][off + i] : make_float4(0.f, 0.f, 0.f, 0.f);
+        for (int i = 0; i < W; ++i) out[i] = s.p[kFirstOut + i] + c * size_t(chunk_vec);
+        float4 v[R][U], nxt[R][U];
+        if (PIPE) load_batch<R, U, T>(v, in, 0, chunk_vec);
+        for (uint32_t base = 0; base < chunk_vec; base += T * U) {   // a run-time bound, as in the kernels
+            if (PIPE) {
+                if (base + T * U < chunk_vec) load_batch<R, U, T>(nxt, in, base + T * U, chunk_vec);
+            } else {
+                load_batch<R, U, T>(v, in, base, chunk_vec);
             }
 #pragma unroll
             for (int u = 0; u < U; ++u) {
-                const int i = base + u * T + threadIdx.x;
+                const uint32_t i = base + u * T + tid;
+                if (i >= chunk_vec) continue;
                 float4 acc = v[0][u];
 #pragma unroll
                 for (int r = 1; r < R; ++r) {
@@ -57,44 +87,61 @@ __global__ void __launch_bounds__(T, 1) walk(Streams s, size_t n_chunks) {
                     acc.z += v[r][u].z;
                     acc.w += v[r][u].w;
                 }
-                if (i < kChunkVec) {
 #pragma unroll
-                    for (int w = 0; w < W; ++w) __stcs(&s.p[R + w][off + i], acc);
-                }
+                for (int w = 0; w < W; ++w) __stcs(&out[w][i], acc);
                 if (W == 0 && acc.x == 12345.678f) s.p[0][0] = acc;   // never true: keeps the loads alive
+            }
+            if (PIPE) {
+#pragma unroll
+                for (int u = 0; u < U; ++u)
+#pragma unroll
+                    for (int r = 0; r < R; ++r) v[r][u] = nxt[r][u];
             }
         }
     }
 }
 
-template <int R, int W, int T, int U>
-int run(size_t n_elems, int ctas_per_sm) {
+template <int R, int W, int T, int U, bool INPLACE = false, bool PIPE = false>
+int run(size_t n_elems, int ctas_per_sm, size_t stagger, bool after_read = false) {
     static_assert(R + W <= kMaxStreams, "too many streams");
+    static_assert(!INPLACE || W <= R, "in place: every result overwrites a stream that was read");
+    static_assert(R >= 2, "the read-only pass walks the first two streams");
+    constexpr int kAlloc = INPLACE ? R : R + W;
     const size_t n_chunks = n_elems / (size_t(kChunkVec) * 4);
     const size_t bytes = n_chunks * size_t(kChunkVec) * sizeof(float4);
     Streams s;
-    for (int i = 0; i < R + W; ++i) {
-        CK(cudaMalloc(&s.p[i], bytes));
-        CK(cudaMemset(s.p[i], 0, bytes));
+    void *base[kMaxStreams];
+    for (int i = 0; i < kAlloc; ++i) {
+        CK(cudaMalloc(&base[i], bytes + stagger * kMaxStreams));
+        CK(cudaMemset(base[i], 0x3c + i, bytes + stagger * kMaxStreams));
+        s.p[i] = reinterpret_cast<float4 *>(static_cast<char *>(base[i]) + stagger * i);
     }
     int sms = 0;
     CK(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, 0));
     cudaEvent_t a, b;
     CK(cudaEventCreate(&a));
     CK(cudaEventCreate(&b));
-    for (int i = 0; i < 3; ++i) walk<R, W, T, U><<<sms * ctas_per_sm, T>>>(s, n_chunks);
-    CK(cudaDeviceSynchronize());
+    // Every timed launch has its own pair of events.  With `after_read` a read-only pass over the
+    // first two streams runs before it (untimed), as the reduction runs before the update in a
+    // step: the timed pass then starts on an L2 full of clean lines instead of the dirty lines its
+    // predecessor left behind.
     const int reps = 10;
-    CK(cudaEventRecord(a));
-    for (int i = 0; i < reps; ++i) walk<R, W, T, U><<<sms * ctas_per_sm, T>>>(s, n_chunks);
-    CK(cudaEventRecord(b));
-    CK(cudaEventSynchronize(b));
-    float ms = 0.f;
-    CK(cudaEventElapsedTime(&ms, a, b));
-    ms /= reps;
-    printf("streams R=%d W=%d T=%d U=%d ctas/sm=%d elems=%zu ms=%.3f GB/s=%.0f\n", R, W, T, U, ctas_per_sm,
-           n_chunks * size_t(kChunkVec) * 4, ms, double(bytes) * (R + W) / (ms * 1e-3) / 1e9);
-    for (int i = 0; i < R + W; ++i) cudaFree(s.p[i]);
+    float total = 0.f;
+    for (int i = 0; i < 3 + reps; ++i) {
+        if (after_read) walk<2, 0, 256, 8, false, false><<<sms * 4, 256>>>(s, n_chunks, kChunkVec);
+        CK(cudaEventRecord(a));
+        walk<R, W, T, U, INPLACE, PIPE><<<sms * ctas_per_sm, T>>>(s, n_chunks, kChunkVec);
+        CK(cudaEventRecord(b));
+        CK(cudaEventSynchronize(b));
+        float ms1 = 0.f;
+        CK(cudaEventElapsedTime(&ms1, a, b));
+        if (i >= 3) total += ms1;
+    }
+    const float ms = total / reps;
+    printf("streams stagger=%zu R=%d W=%d place=%s after=%s pipelined=%s T=%d U=%d ctas/sm=%d elems=%zu ms=%.3f GB/s=%.0f\n", stagger, R, W,
+           INPLACE ? "in" : "out", after_read ? "read" : "same", PIPE ? "yes" : "no", T, U, ctas_per_sm, n_chunks * size_t(kChunkVec) * 4, ms,
+           double(bytes) * (R + W) / (ms * 1e-3) / 1e9);
+    for (int i = 0; i < kAlloc; ++i) cudaFree(base[i]);
     cudaEventDestroy(a);
     cudaEventDestroy(b);
     return 0;
@@ -106,20 +153,53 @@ int main(int argc, char **argv) {
         fprintf(stderr, "elements per stream must lie in [2^24, 2^31]\n");
         return 2;
     }
+    const size_t g = argc > 2 ? strtoull(argv[2], nullptr, 10) : 0;
+    if (g % 16 || g > (size_t(1) << 24)) {
+        fprintf(stderr, "stagger must be a multiple of 16 bytes, at most 2^24\n");
+        return 2;
+    }
     int rc = 0;
-    rc |= run<1, 1, 256, 8>(n, 1);
-    rc |= run<1, 1, 256, 8>(n, 4);
-    rc |= run<2, 0, 256, 8>(n, 4);
-    rc |= run<2, 2, 256, 8>(n, 1);
-    rc |= run<2, 2, 512, 4>(n, 1);
-    rc |= run<2, 2, 256, 4>(n, 4);
-    rc |= run<2, 1, 512, 4>(n, 1);
-    rc |= run<5, 4, 1024, 1>(n, 1);
-    rc |= run<5, 4, 896, 1>(n, 1);
-    rc |= run<5, 4, 640, 1>(n, 1);
-    rc |= run<5, 4, 512, 2>(n, 1);
-    rc |= run<5, 4, 256, 2>(n, 2);
-    rc |= run<5, 4, 256, 1>(n, 4);
-    rc |= run<5, 3, 896, 1>(n, 1);
+    rc |= run<2, 1, 256, 8>(n, 4, g);
+    rc |= run<2, 0, 256, 8>(n, 4, g);
+    rc |= run<2, 2, 256, 8>(n, 1, g);
+    rc |= run<2, 2, 512, 4>(n, 1, g);
+    rc |= run<2, 2, 256, 4>(n, 4, g);
+    rc |= run<2, 1, 512, 4>(n, 1, g);
+    rc |= run<5, 4, 1024, 1>(n, 1, g);
+    rc |= run<5, 4, 896, 1>(n, 1, g);
+    rc |= run<5, 4, 640, 1>(n, 1, g);
+    rc |= run<5, 4, 512, 2>(n, 1, g);
+    rc |= run<5, 4, 256, 2>(n, 2, g);
+    rc |= run<5, 4, 256, 1>(n, 4, g);
+    rc |= run<5, 3, 896, 1>(n, 1, g);
+    // the same mixes with the results written over the streams that were read
+    rc |= run<2, 2, 256, 8, true>(n, 1, g);
+    rc |= run<2, 2, 512, 4, true>(n, 1, g);
+    rc |= run<5, 4, 1024, 1, true>(n, 1, g);
+    rc |= run<5, 4, 896, 1, true>(n, 1, g);
+    rc |= run<5, 4, 640, 1, true>(n, 1, g);
+    rc |= run<5, 4, 512, 2, true>(n, 1, g);
+    rc |= run<5, 4, 256, 2, true>(n, 2, g);
+    rc |= run<5, 4, 256, 4, true>(n, 1, g);
+    rc |= run<5, 3, 896, 1, true>(n, 1, g);
+    // ... with the next batch's loads issued before the current batch's stores
+    rc |= run<2, 2, 256, 8, true, true>(n, 1, g);
+    rc |= run<2, 2, 256, 4, true, true>(n, 1, g);
+    rc |= run<2, 2, 512, 4, true, true>(n, 1, g);
+    rc |= run<5, 4, 1024, 1, true, true>(n, 1, g);
+    rc |= run<5, 4, 896, 1, true, true>(n, 1, g);
+    rc |= run<5, 4, 640, 1, true, true>(n, 1, g);
+    rc |= run<5, 4, 512, 1, true, true>(n, 1, g);
+    rc |= run<5, 4, 512, 2, true, true>(n, 1, g);
+    rc |= run<5, 4, 256, 2, true, true>(n, 1, g);
+    rc |= run<5, 4, 256, 2, true, true>(n, 2, g);
+    rc |= run<5, 4, 256, 4, true, true>(n, 1, g);
+    // ... and each such pass after a read-only pass, as in a step
+    rc |= run<2, 2, 256, 8, true>(n, 1, g, true);
+    rc |= run<2, 2, 512, 4, true>(n, 1, g, true);
+    rc |= run<2, 1, 512, 4>(n, 1, g, true);
+    rc |= run<5, 4, 896, 1, true>(n, 1, g, true);
+    rc |= run<5, 4, 640, 1, true>(n, 1, g, true);
+    rc |= run<5, 4, 256, 2, true>(n, 2, g, true);
     return rc;
 }
