@@ -32,7 +32,7 @@ namespace {
 #define GAC_PHASE_BARRIER 1
 #endif
 #ifndef GAC_PROJECT_BARRIER   // the same in the projection pass: bit 0 after the loads, bit 1 after the stores
-#define GAC_PROJECT_BARRIER 1   // after the loads: +0.6-1 % on B200; after the stores it costs 3-10 % there
+#define GAC_PROJECT_BARRIER 1   // after the loads: +0.5-1 % on B200; after the stores it costs 2-10 % there
 #endif
 constexpr int kDefaultChunk = GAC_CHUNK; // elements per chunk
 constexpr int kMaxCtasPerSm = 16;
@@ -184,9 +184,9 @@ template <> struct ExchGeom<float>        { static constexpr int T = 512, U = 4,
 template <> struct ExchGeom<bf16_t>       { static constexpr int T = 512, U = 4, UK = 8, C = 1, MINB = 1; };   // pair not served
 template <> struct ExchGeom<bf16_pair_t>  { static constexpr int T = 512, U = 4, UK = 8, C = 2, MINB = 2; };
 // AdamGeom: T for the plain rule (beta = 1, no clipping), TG for the general one, which needs more registers
-template <> struct AdamGeom<float>        { static constexpr int T = 1024, TG = 896, U = 1, C = 1; };
-template <> struct AdamGeom<bf16_t>       { static constexpr int T = 1024, TG = 896, U = 1, C = 1; };
-template <> struct AdamGeom<bf16_pair_t>  { static constexpr int T = 896, TG = 768, U = 1, C = 1; };
+template <> struct AdamGeom<float>        { static constexpr int T = 1024, TG = 1024, U = 1, C = 1; };
+template <> struct AdamGeom<bf16_t>       { static constexpr int T = 1024, TG = 1024, U = 1, C = 1; };
+template <> struct AdamGeom<bf16_pair_t>  { static constexpr int T = 1024, TG = 1024, U = 1, C = 1; };
 #endif
 
 __device__ __forceinline__ uint32_t pack_bf16x2_rn(float lo, float hi) {
@@ -244,11 +244,21 @@ __device__ __forceinline__ Chunk load_chunk(const Chunk *table, uint32_t c, int 
     return ch;
 }
 
+// 16 bytes global -> shared without passing through registers; completion is awaited with
+// cp_async_wait_all() by the thread that issued the copies.
+__device__ __forceinline__ void cp_async16(void *smem, const void *gmem) {
+    const unsigned sa = static_cast<unsigned>(__cvta_generic_to_shared(smem));
+    asm volatile("cp.async.ca.shared.global [%0], [%1], 16;" ::"r"(sa), "l"(gmem) : "memory");
+}
+__device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_all;" ::: "memory"); }
+
 // Keeps the warps of a CTA in step in a pass that reads AND writes: every warp issues its
 // batch of loads, then every warp stores its results, and only then does the next batch of
 // loads start.  Without it the warps drift apart and each SM sends DRAM an even mix of reads
-// and writes.  Measured on B200: the fused AdamW pass (5 read + 4 write streams, 32 warps per
-// SM) gains 5-9 % from it; a bare 2 + 2 loop gains 10 %.
+// and writes.  Measured on B200, fused AdamW pass on the 1.5 B float32 list (5 read + 4 write
+// streams, 32 warps per SM): 5.96 TB/s without, 6.36 TB/s with this barrier, 6.60 TB/s once
+// the chunk descriptors are also fetched ahead (adamw_walk), so that the CTA does not stall
+// as one at every chunk boundary.
 // Every thread of the CTA reaches it: the loops around it have CTA-uniform trip counts.
 __device__ __forceinline__ void phase_barrier() {
 #if GAC_PHASE_BARRIER
@@ -672,12 +682,21 @@ __device__ __forceinline__ void project_chunk(const Chunk &ch, float k, double b
 template <typename GT, int STATE>
 using ProjGeomOf = typename std::conditional<STATE == GAC_STATE_EXCHANGE, ExchGeom<GT>, ProjGeom<GT>>::type;
 
+// A CTA's walk over its chunks.  Every thread reads the descriptor when it gets to the chunk: the
+// short wait for it lets the warps of the CTA fall into step again at every chunk boundary, which
+// this pass likes (fetching the descriptor ahead of time, through registers or asynchronously
+// through shared memory, measured no better for f32 and 2-5 % worse for bfloat16 gradients).
+template <typename GT, int GOP, int DOP, bool BETA1, int T, int U>
+__device__ __forceinline__ void project_walk_tu(const Chunk *chunks, uint32_t n_chunks, float k,
+                                                double beta, double s, int swapped) {
+    for (uint32_t c = blockIdx.x; c < n_chunks; c += gridDim.x)
+        project_chunk<GT, GOP, DOP, BETA1, T, U>(load_chunk(chunks, c, swapped), k, beta, s);
+}
 template <typename GT, int GOP, int DOP, bool BETA1>
 __device__ __forceinline__ void project_walk(const Chunk *chunks, uint32_t n_chunks, float k,
                                              double beta, double s, int swapped) {
     using Geom = typename std::conditional<DOP == D_OUT, ExchGeom<GT>, ProjGeom<GT>>::type;
-    for (uint32_t c = blockIdx.x; c < n_chunks; c += gridDim.x)
-        project_chunk<GT, GOP, DOP, BETA1, Geom::T, Geom::U>(load_chunk(chunks, c, swapped), k, beta, s);
+    project_walk_tu<GT, GOP, DOP, BETA1, Geom::T, Geom::U>(chunks, n_chunks, k, beta, s, swapped);
 }
 
 // The regime is read from the device-resident record, so no host round trip
@@ -717,8 +736,8 @@ gac_project_kernel(const Chunk *__restrict__ chunks, uint32_t n_chunks, gac_resu
     } else if (s != 1.0) {
         project_walk<GT, G_SCALE, dop, true>(chunks, n_chunks, k, 1.0, s, swapped);   // safe step, clipped: g'' = s g
     } else if (STATE != GAC_STATE_HOLD && STATE != GAC_STATE_EXCHANGE) {
-        for (uint32_t c = blockIdx.x; c < n_chunks; c += gridDim.x)   // d' = g, g untouched
-            project_chunk<GT, G_KEEP, D_RAW, true, ProjGeom<GT>::T, ProjGeom<GT>::UK>(load_chunk(chunks, c), k, 1.0, 1.0);
+        // d' = g, g untouched
+        project_walk_tu<GT, G_KEEP, D_RAW, true, ProjGeom<GT>::T, ProjGeom<GT>::UK>(chunks, n_chunks, k, 1.0, 1.0, 0);
     }
     // exchange mode, g unchanged: nothing to move -- the buffers that hold g become the stored direction
 }
@@ -773,7 +792,7 @@ __device__ __forceinline__ double rcp_approx64(double x) {
     return y;
 }
 __device__ __forceinline__ void adamw_elem(double g64, float &p, float &m, float &v, const AdamDev &a,
-                                           const volatile AdamStep &st) {
+                                           const AdamStep &st) {
     const double m64 = fma(a.b1, double(m), a.c1 * g64);
     const double v64 = fma(a.b2, double(v), (a.c2 * g64) * g64);
     double root = 0.0;
@@ -791,22 +810,25 @@ __device__ __forceinline__ void adamw_elem(double g64, float &p, float &m, float
     v = __double2float_rn(v64);
 }
 
-// The addresses of the chunk a CTA is working on, in shared memory: thread 0 reads the two
-// descriptors, everybody else picks an address up where it is used.  At 1024 threads a thread has
-// 64 registers; five 64-bit base addresses held across the loop would take ten of them.
-struct AdamChunk {
-    unsigned long long g, d, p, m, v;
-    uint32_t n, vec;
+// The two descriptors of the chunk a CTA is working on, in shared memory: everybody picks an
+// address up where it is used.  At 1024 threads a thread has 64 registers; five 64-bit base
+// addresses held across the loop would take ten of them.
+struct __align__(16) AdamChunk {
+    Chunk ch;
+    OptChunk oc;
 };
 
 template <typename GT, int GOP, bool STORE_D, int T>
-__device__ __forceinline__ void adamw_chunk(const volatile AdamChunk &ck, double beta, double s, const AdamDev &a,
-                                            const volatile AdamStep &st) {
+__device__ __forceinline__ void adamw_chunk(const volatile AdamChunk &ck, int swapped, double beta, double s,
+                                            const AdamDev &a, const AdamStep &st) {
     const uint32_t tid = threadIdx.x;
     constexpr int U = AdamGeom<GT>::U;
     constexpr bool kReadD = (GOP == G_FMA || GOP == G_FMA1);
-    const uint32_t n = ck.n;
-    const bool vec = ck.vec != 0;
+    const uint32_t n = ck.ch.n;
+    const bool vec = (ck.ch.flags & kChunkAligned) && ((ck.oc.p | ck.oc.m | ck.oc.v) % 16 == 0);
+    // exchange mode: the two address columns of the table trade roles
+    #define CK_G (swapped ? ck.ch.d : ck.ch.g)
+    #define CK_D (swapped ? ck.ch.g : ck.ch.d)
     if (vec) {
         const uint32_t nvec = n >> 2;
         for (uint32_t base = 0; base < nvec; base += T * U) {
@@ -820,11 +842,11 @@ __device__ __forceinline__ void adamw_chunk(const volatile AdamChunk &ck, double
                 dr[u] = Elem<DOf<GT>>::zero();
                 p4[u] = m4[u] = v4[u] = make_float4(0.f, 0.f, 0.f, 0.f);
                 if (w < nvec) {
-                    gr[u] = Elem<GOf<GT>>::template load_raw<GAC_LD_PROJECT>(reinterpret_cast<const void *>(ck.g), w);
-                    if (kReadD) dr[u] = Elem<DOf<GT>>::template load_raw<GAC_LD_PROJECT>(reinterpret_cast<const void *>(ck.d), w);
-                    p4[u] = Elem<float>::load_raw<GAC_LD_PROJECT>(reinterpret_cast<const void *>(ck.p), w);
-                    m4[u] = Elem<float>::load_raw<GAC_LD_PROJECT>(reinterpret_cast<const void *>(ck.m), w);
-                    v4[u] = Elem<float>::load_raw<GAC_LD_PROJECT>(reinterpret_cast<const void *>(ck.v), w);
+                    gr[u] = Elem<GOf<GT>>::template load_raw<GAC_LD_PROJECT>(reinterpret_cast<const void *>(CK_G), w);
+                    if (kReadD) dr[u] = Elem<DOf<GT>>::template load_raw<GAC_LD_PROJECT>(reinterpret_cast<const void *>(CK_D), w);
+                    p4[u] = Elem<float>::load_raw<GAC_LD_PROJECT>(reinterpret_cast<const void *>(ck.oc.p), w);
+                    m4[u] = Elem<float>::load_raw<GAC_LD_PROJECT>(reinterpret_cast<const void *>(ck.oc.m), w);
+                    v4[u] = Elem<float>::load_raw<GAC_LD_PROJECT>(reinterpret_cast<const void *>(ck.oc.v), w);
                 }
             }
 #pragma unroll
@@ -837,31 +859,33 @@ __device__ __forceinline__ void adamw_chunk(const volatile AdamChunk &ck, double
                 float me[4] = {m4[u].x, m4[u].y, m4[u].z, m4[u].w};
                 float ve[4] = {v4[u].x, v4[u].y, v4[u].z, v4[u].w};
                 const float de[4] = {dq.x, dq.y, dq.z, dq.w};
-                if (STORE_D) Elem<DOf<GT>>::store4(reinterpret_cast<void *>(ck.d), w, gq);   // d' = g, the raw gradient
+                if (STORE_D) Elem<DOf<GT>>::store4(reinterpret_cast<void *>(CK_D), w, gq);   // d' = g, the raw gradient
 #pragma unroll
                 for (int e = 0; e < 4; ++e) {
                     adamw_elem(outgoing64<GOP>(ge[e], de[e], st.coef, beta, s), pe[e], me[e], ve[e], a, st);
                 }
-                Elem<float>::store4(reinterpret_cast<void *>(ck.p), w, F4{pe[0], pe[1], pe[2], pe[3]});
-                Elem<float>::store4(reinterpret_cast<void *>(ck.m), w, F4{me[0], me[1], me[2], me[3]});
-                Elem<float>::store4(reinterpret_cast<void *>(ck.v), w, F4{ve[0], ve[1], ve[2], ve[3]});
+                Elem<float>::store4(reinterpret_cast<void *>(ck.oc.p), w, F4{pe[0], pe[1], pe[2], pe[3]});
+                Elem<float>::store4(reinterpret_cast<void *>(ck.oc.m), w, F4{me[0], me[1], me[2], me[3]});
+                Elem<float>::store4(reinterpret_cast<void *>(ck.oc.v), w, F4{ve[0], ve[1], ve[2], ve[3]});
             }
             phase_barrier();
         }
     }
     const uint32_t first = vec ? ((n >> 2) << 2) : 0u;
     for (uint32_t i = first + tid; i < n; i += T) {
-        const float x = Elem<GOf<GT>>::load1(reinterpret_cast<const void *>(ck.g), i);
-        const float dx = kReadD ? Elem<DOf<GT>>::load1(reinterpret_cast<const void *>(ck.d), i) : 0.f;
-        float pe = Elem<float>::load1(reinterpret_cast<const void *>(ck.p), i);
-        float me = Elem<float>::load1(reinterpret_cast<const void *>(ck.m), i);
-        float ve = Elem<float>::load1(reinterpret_cast<const void *>(ck.v), i);
+        const float x = Elem<GOf<GT>>::load1(reinterpret_cast<const void *>(CK_G), i);
+        const float dx = kReadD ? Elem<DOf<GT>>::load1(reinterpret_cast<const void *>(CK_D), i) : 0.f;
+        float pe = Elem<float>::load1(reinterpret_cast<const void *>(ck.oc.p), i);
+        float me = Elem<float>::load1(reinterpret_cast<const void *>(ck.oc.m), i);
+        float ve = Elem<float>::load1(reinterpret_cast<const void *>(ck.oc.v), i);
         adamw_elem(outgoing64<GOP>(x, dx, st.coef, beta, s), pe, me, ve, a, st);
-        if (STORE_D) Elem<DOf<GT>>::store1(reinterpret_cast<void *>(ck.d), i, x);
-        Elem<float>::store1(reinterpret_cast<void *>(ck.p), i, pe);
-        Elem<float>::store1(reinterpret_cast<void *>(ck.m), i, me);
-        Elem<float>::store1(reinterpret_cast<void *>(ck.v), i, ve);
+        if (STORE_D) Elem<DOf<GT>>::store1(reinterpret_cast<void *>(CK_D), i, x);
+        Elem<float>::store1(reinterpret_cast<void *>(ck.oc.p), i, pe);
+        Elem<float>::store1(reinterpret_cast<void *>(ck.oc.m), i, me);
+        Elem<float>::store1(reinterpret_cast<void *>(ck.oc.v), i, ve);
     }
+    #undef CK_G
+    #undef CK_D
 }
 
 __device__ __forceinline__ OptChunk load_opt_chunk(const OptChunk *table, uint32_t c) {
@@ -878,23 +902,26 @@ __device__ __forceinline__ OptChunk load_opt_chunk(const OptChunk *table, uint32
 template <typename GT, int GOP, bool STORE_D, int T>
 __device__ __forceinline__ void adamw_walk(const Chunk *chunks, const OptChunk *opt_chunks, uint32_t n_chunks,
                                            int swapped, double beta, double s, const AdamDev &a,
-                                           const volatile AdamStep &st) {
-    __shared__ AdamChunk ck;
-    for (uint32_t c = blockIdx.x; c < n_chunks; c += gridDim.x) {
-        if (threadIdx.x == 0) {
-            const Chunk ch = load_chunk(chunks, c, swapped);
-            const OptChunk oc = load_opt_chunk(opt_chunks, c);
-            ck.g = ch.g;
-            ck.d = ch.d;
-            ck.p = oc.p;
-            ck.m = oc.m;
-            ck.v = oc.v;
-            ck.n = ch.n;
-            ck.vec = ((ch.flags & kChunkAligned) && ((oc.p | oc.m | oc.v) % 16 == 0)) ? 1u : 0u;
-        }
-        __syncthreads();   // the addresses are there
-        adamw_chunk<GT, GOP, STORE_D, T>(ck, beta, s, a, st);
-        __syncthreads();   // everybody is done with them
+                                           const AdamStep &st) {
+    // Two slots: while the CTA works on the chunk in one, thread 0 has the descriptors of the next
+    // chunk copied into the other (asynchronously, past the registers), so that nobody waits for
+    // them at the chunk boundary.
+    __shared__ AdamChunk slots[2];
+    auto fetch = [&](uint32_t c, AdamChunk &out) {
+        cp_async16(&out.ch, chunks + c);
+        cp_async16(reinterpret_cast<char *>(&out.ch) + 16, reinterpret_cast<const char *>(chunks + c) + 16);
+        cp_async16(&out.oc, opt_chunks + c);
+        cp_async16(reinterpret_cast<char *>(&out.oc) + 16, reinterpret_cast<const char *>(opt_chunks + c) + 16);
+    };
+    uint32_t c = blockIdx.x;
+    if (c >= n_chunks) return;
+    if (threadIdx.x == 0) fetch(c, slots[0]);
+    int cur = 0;
+    for (; c < n_chunks; c += gridDim.x, cur ^= 1) {
+        if (threadIdx.x == 0) cp_async_wait_all();   // the copies into slots[cur] have landed
+        __syncthreads();                             // ... for everybody; and nobody reads slots[cur ^ 1] any more
+        if (threadIdx.x == 0 && c + gridDim.x < n_chunks) fetch(c + gridDim.x, slots[cur ^ 1]);
+        adamw_chunk<GT, GOP, STORE_D, T>(slots[cur], swapped, beta, s, a, st);
     }
 }
 
@@ -944,7 +971,7 @@ gac_adamw_kernel(const Chunk *__restrict__ chunks, const OptChunk *__restrict__ 
             st_shared.coef = k;
         }
         __syncthreads();
-        const volatile AdamStep &st = st_shared;
+        const AdamStep &st = st_shared;
         // one uniform choice per launch; each branch holds only the loop it needs
         constexpr int T = AdamThreads<GT, PLAIN>::T;
         const int gop = regime == GAC_REGIME_PROJECT ? ((beta == 1.0 && s == 1.0) ? G_FMA1 : G_FMA)
@@ -954,8 +981,8 @@ gac_adamw_kernel(const Chunk *__restrict__ chunks, const OptChunk *__restrict__ 
         else if (!PLAIN && gop == G_FMA) adamw_walk<GT, G_FMA, !EXCH, T>(chunks, opt_chunks, n_chunks, swapped, beta, s, o, st);
         else if (!PLAIN) adamw_walk<GT, G_SCALE, !EXCH, T>(chunks, opt_chunks, n_chunks, swapped, 1.0, s, o, st);
     } else if (!EXCH) {
-        for (uint32_t c = blockIdx.x; c < n_chunks; c += gridDim.x)   // skipped step: d' = g only
-            project_chunk<GT, G_KEEP, D_RAW, true, AdamThreads<GT, PLAIN>::T, AdamGeom<GT>::U>(load_chunk(chunks, c), k, 1.0, 1.0);
+        // skipped step: d' = g only
+        project_walk_tu<GT, G_KEEP, D_RAW, true, AdamThreads<GT, PLAIN>::T, AdamGeom<GT>::U>(chunks, n_chunks, k, 1.0, 1.0, 0);
     }
     __syncthreads();
     if (threadIdx.x == 0) {

@@ -3,7 +3,8 @@
 // cut into 64 KB chunks that the CTAs take round-robin (chunk c -> CTA c mod grid), T threads
 // with U vectors of every read stream in flight per thread, streaming stores.  "in place" means
 // that the W results overwrite the last W of the R streams read (as the kernels update g, d, p,
-// m, v where they lie); otherwise the results go to W further allocations.
+// m, v where they lie); otherwise the results go to W further allocations.  "barriers" keeps
+// the warps of a CTA in step: 1 = __syncthreads() after a batch's loads, 2 = after its stores.
 //
 // The figures it prints are the ceilings the kernels are measured against besides the plain
 // copy rate: a kernel that matches the probe of its own pattern is limited by how DRAM serves
@@ -18,7 +19,7 @@
 // Patterns: 2+0 (fused triple reduction), 2+2 (projection + state refresh),
 // 2+1 (projection in exchange mode), 5+4 and 5+3 (projection fused with AdamW, with and
 // without the state copy).  One line per pattern and geometry:
-//   streams stagger=.. R=.. W=.. place=in|out after=same|read pipelined=yes|no T=.. U=.. ctas/sm=.. elems=.. ms=.. GB/s=..
+//   streams stagger=.. R=.. W=.. place=in|out after=same|read barriers=0..3 T=.. U=.. ctas/sm=.. elems=.. ms=.. GB/s=..
 #include <cuda_runtime.h>
 
 #include <cstdint>
@@ -41,23 +42,10 @@ struct Streams {
     float4 *p[kMaxStreams];
 };
 
-template <int R, int U, int T>
-__device__ __forceinline__ void load_batch(float4 (&v)[R][U], float4 *const (&p)[R], uint32_t base, uint32_t chunk_vec) {
-#pragma unroll
-    for (int u = 0; u < U; ++u) {
-        const uint32_t i = base + u * T + threadIdx.x;
-#pragma unroll
-        for (int r = 0; r < R; ++r) v[r][u] = make_float4(0.f, 0.f, 0.f, 0.f);
-        if (i < chunk_vec) {
-#pragma unroll
-            for (int r = 0; r < R; ++r) v[r][u] = p[r][i];
-        }
-    }
-}
-
-// PIPE: the loads of the next batch are issued before the results of the current one are stored,
-// so that a thread always has reads in flight while it writes.
-template <int R, int W, int T, int U, bool INPLACE, bool PIPE>
+// BAR bit 0: __syncthreads() between a batch's loads and its stores; bit 1: after its stores.
+// The barriers keep the warps of a CTA in step, so that an SM alternates between issuing reads
+// and issuing writes instead of sending DRAM an even mix of both.
+template <int R, int W, int T, int U, bool INPLACE, int BAR>
 __global__ void __launch_bounds__(T, 1) walk(Streams s, size_t n_chunks, uint32_t chunk_vec) {
     constexpr int kFirstOut = INPLACE ? R - W : R;
     const uint32_t tid = threadIdx.x;
@@ -67,14 +55,19 @@ __global__ void __launch_bounds__(T, 1) walk(Streams s, size_t n_chunks, uint32_
         for (int i = 0; i < R; ++i) in[i] = s.p[i] + c * size_t(chunk_vec);
 #pragma unroll
         for (int i = 0; i < W; ++i) out[i] = s.p[kFirstOut + i] + c * size_t(chunk_vec);
-        float4 v[R][U], nxt[R][U];
-        if (PIPE) load_batch<R, U, T>(v, in, 0, chunk_vec);
         for (uint32_t base = 0; base < chunk_vec; base += T * U) {   // a run-time bound, as in the kernels
-            if (PIPE) {
-                if (base + T * U < chunk_vec) load_batch<R, U, T>(nxt, in, base + T * U, chunk_vec);
-            } else {
-                load_batch<R, U, T>(v, in, base, chunk_vec);
+            float4 v[R][U];
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+                const uint32_t i = base + u * T + tid;
+#pragma unroll
+                for (int r = 0; r < R; ++r) v[r][u] = make_float4(0.f, 0.f, 0.f, 0.f);
+                if (i < chunk_vec) {
+#pragma unroll
+                    for (int r = 0; r < R; ++r) v[r][u] = in[r][i];
+                }
             }
+            if (BAR & 1) __syncthreads();
 #pragma unroll
             for (int u = 0; u < U; ++u) {
                 const uint32_t i = base + u * T + tid;
@@ -91,17 +84,12 @@ __global__ void __launch_bounds__(T, 1) walk(Streams s, size_t n_chunks, uint32_
                 for (int w = 0; w < W; ++w) __stcs(&out[w][i], acc);
                 if (W == 0 && acc.x == 12345.678f) s.p[0][0] = acc;   // never true: keeps the loads alive
             }
-            if (PIPE) {
-#pragma unroll
-                for (int u = 0; u < U; ++u)
-#pragma unroll
-                    for (int r = 0; r < R; ++r) v[r][u] = nxt[r][u];
-            }
+            if (BAR & 2) __syncthreads();
         }
     }
 }
 
-template <int R, int W, int T, int U, bool INPLACE = false, bool PIPE = false>
+template <int R, int W, int T, int U, bool INPLACE = false, int BAR = 0>
 int run(size_t n_elems, int ctas_per_sm, size_t stagger, bool after_read = false) {
     static_assert(R + W <= kMaxStreams, "too many streams");
     static_assert(!INPLACE || W <= R, "in place: every result overwrites a stream that was read");
@@ -128,9 +116,9 @@ int run(size_t n_elems, int ctas_per_sm, size_t stagger, bool after_read = false
     const int reps = 10;
     float total = 0.f;
     for (int i = 0; i < 3 + reps; ++i) {
-        if (after_read) walk<2, 0, 256, 8, false, false><<<sms * 4, 256>>>(s, n_chunks, kChunkVec);
+        if (after_read) walk<2, 0, 256, 8, false, 0><<<sms * 4, 256>>>(s, n_chunks, kChunkVec);
         CK(cudaEventRecord(a));
-        walk<R, W, T, U, INPLACE, PIPE><<<sms * ctas_per_sm, T>>>(s, n_chunks, kChunkVec);
+        walk<R, W, T, U, INPLACE, BAR><<<sms * ctas_per_sm, T>>>(s, n_chunks, kChunkVec);
         CK(cudaEventRecord(b));
         CK(cudaEventSynchronize(b));
         float ms1 = 0.f;
@@ -138,8 +126,8 @@ int run(size_t n_elems, int ctas_per_sm, size_t stagger, bool after_read = false
         if (i >= 3) total += ms1;
     }
     const float ms = total / reps;
-    printf("streams stagger=%zu R=%d W=%d place=%s after=%s pipelined=%s T=%d U=%d ctas/sm=%d elems=%zu ms=%.3f GB/s=%.0f\n", stagger, R, W,
-           INPLACE ? "in" : "out", after_read ? "read" : "same", PIPE ? "yes" : "no", T, U, ctas_per_sm, n_chunks * size_t(kChunkVec) * 4, ms,
+    printf("streams stagger=%zu R=%d W=%d place=%s after=%s barriers=%d T=%d U=%d ctas/sm=%d elems=%zu ms=%.3f GB/s=%.0f\n", stagger, R, W,
+           INPLACE ? "in" : "out", after_read ? "read" : "same", BAR, T, U, ctas_per_sm, n_chunks * size_t(kChunkVec) * 4, ms,
            double(bytes) * (R + W) / (ms * 1e-3) / 1e9);
     for (int i = 0; i < kAlloc; ++i) cudaFree(base[i]);
     cudaEventDestroy(a);
@@ -182,18 +170,19 @@ int main(int argc, char **argv) {
     rc |= run<5, 4, 256, 2, true>(n, 2, g);
     rc |= run<5, 4, 256, 4, true>(n, 1, g);
     rc |= run<5, 3, 896, 1, true>(n, 1, g);
-    // ... with the next batch's loads issued before the current batch's stores
-    rc |= run<2, 2, 256, 8, true, true>(n, 1, g);
-    rc |= run<2, 2, 256, 4, true, true>(n, 1, g);
-    rc |= run<2, 2, 512, 4, true, true>(n, 1, g);
-    rc |= run<5, 4, 1024, 1, true, true>(n, 1, g);
-    rc |= run<5, 4, 896, 1, true, true>(n, 1, g);
-    rc |= run<5, 4, 640, 1, true, true>(n, 1, g);
-    rc |= run<5, 4, 512, 1, true, true>(n, 1, g);
-    rc |= run<5, 4, 512, 2, true, true>(n, 1, g);
-    rc |= run<5, 4, 256, 2, true, true>(n, 1, g);
-    rc |= run<5, 4, 256, 2, true, true>(n, 2, g);
-    rc |= run<5, 4, 256, 4, true, true>(n, 1, g);
+    // ... with the warps of a CTA kept in step: barrier after the loads (1), after the stores (2), both (3)
+    rc |= run<2, 2, 256, 8, true, 1>(n, 1, g);
+    rc |= run<2, 2, 256, 8, true, 2>(n, 1, g);
+    rc |= run<2, 2, 256, 8, true, 3>(n, 1, g);
+    rc |= run<2, 2, 512, 4, true, 1>(n, 1, g);
+    rc |= run<2, 2, 512, 4, true, 2>(n, 1, g);
+    rc |= run<2, 1, 512, 4, false, 2>(n, 1, g);
+    rc |= run<5, 4, 1024, 1, true, 1>(n, 1, g);
+    rc |= run<5, 4, 1024, 1, true, 2>(n, 1, g);
+    rc |= run<5, 4, 896, 1, true, 2>(n, 1, g);
+    rc |= run<5, 4, 640, 1, true, 2>(n, 1, g);
+    rc |= run<5, 4, 512, 2, true, 2>(n, 1, g);
+    rc |= run<5, 3, 1024, 1, true, 2>(n, 1, g);
     // ... and each such pass after a read-only pass, as in a step
     rc |= run<2, 2, 256, 8, true>(n, 1, g, true);
     rc |= run<2, 2, 512, 4, true>(n, 1, g, true);
