@@ -144,6 +144,16 @@ def recorded_traffic(kernel: str):
         return None
 
 
+def reserve_stdout():
+    """Keeps the process's stdout for the one JSON line: returns a file on a duplicate of it and
+    points descriptor 1 at stderr, so that what libraries print on stdout (NCCL prints its version
+    there) still appears, but not in front of the line."""
+    sys.stdout.flush()
+    line_out = os.fdopen(os.dup(1), "w")
+    os.dup2(2, 1)
+    return line_out
+
+
 # ------------------------------------------------------------------ launcher
 
 def free_port() -> int:
@@ -744,6 +754,7 @@ def main():
 
     from paper_2603_01501_b200 import binding as gb
     gb.load_library()
+    line_out = reserve_stdout()
 
     world = int(os.environ.get("WORLD_SIZE", "1"))
     rank = int(os.environ.get("RANK", "0"))
@@ -865,7 +876,8 @@ def main():
         torch.distributed.barrier()
         torch.distributed.destroy_process_group()
     if rank == 0:
-        print(json.dumps(line))
+        line_out.write(json.dumps(line) + "\n")
+        line_out.flush()
     return 0
 
 
