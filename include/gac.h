@@ -39,7 +39,7 @@ typedef enum {
     GAC_ERR_STATE = 4,         /* calls out of order (project without stats, step going back)*/
     GAC_ERR_NONFINITE = 5,     /* NaN/Inf met in g or d; the step is reported as a violation  */
     GAC_ERR_TIMEOUT = 6        /* gac_decide_exchange: a peer's sums did not arrive within the limit
-                                  (the only wait in this library, bounded)                      */
+                                  (the only wait for another party in this library, bounded)    */
 } gac_status;
 
 typedef enum { GAC_F32 = 0, GAC_BF16 = 1 } gac_dtype;
