@@ -183,10 +183,13 @@ template <> struct ProjGeom<bf16_pair_t>  { static constexpr int T = 512, U = 8,
 template <> struct ExchGeom<float>        { static constexpr int T = 512, U = 4, UK = 8, C = 1, MINB = 1; };
 template <> struct ExchGeom<bf16_t>       { static constexpr int T = 512, U = 4, UK = 8, C = 1, MINB = 1; };   // pair not served
 template <> struct ExchGeom<bf16_pair_t>  { static constexpr int T = 512, U = 4, UK = 8, C = 2, MINB = 2; };
-// AdamGeom: T for the plain rule (beta = 1, no clipping), TG for the general one, which needs more registers
+// AdamGeom: T threads for the plain rule (beta = 1, no clipping), TG for the general one, C CTAs per SM.
+// float32 gradients: one CTA of 1024 threads (a 64 KB chunk is exactly four batches); bfloat16
+// gradients move fewer bytes per batch, and two CTAs of 512 threads, each in step with itself
+// only, overlap one CTA's arithmetic with the other's memory phase (+5-7 % there, -3 % for float32).
 template <> struct AdamGeom<float>        { static constexpr int T = 1024, TG = 1024, U = 1, C = 1; };
-template <> struct AdamGeom<bf16_t>       { static constexpr int T = 1024, TG = 1024, U = 1, C = 1; };
-template <> struct AdamGeom<bf16_pair_t>  { static constexpr int T = 1024, TG = 1024, U = 1, C = 1; };
+template <> struct AdamGeom<bf16_t>       { static constexpr int T = 512, TG = 512, U = 1, C = 2; };
+template <> struct AdamGeom<bf16_pair_t>  { static constexpr int T = 512, TG = 512, U = 1, C = 2; };
 #endif
 
 __device__ __forceinline__ uint32_t pack_bf16x2_rn(float lo, float hi) {
