@@ -18,7 +18,7 @@ from oracle import gac_oracle as orc
 from paper_2603_01501_b200 import binding as gb
 from paper_2603_01501_b200 import synth
 
-from gpu_util import check_decision, check_sums, max_ulp, to_orc_hp
+from gpu_util import check_decision, check_sums, max_ulp, ordered_int, to_orc_hp
 
 pytestmark = pytest.mark.gpu
 
@@ -31,7 +31,7 @@ SLICE = 4 << 20
 def oracle_sums_streamed(g_list, d_list, first_step=False):
     big = max(t.numel() for t in g_list)
     stage_g = torch.empty(big, dtype=g_list[0].dtype, pin_memory=True)
-    stage_d = torch.empty(big, dtype=torch.float32, pin_memory=True)
+    stage_d = torch.empty(big, dtype=d_list[0].dtype, pin_memory=True)
     acc = orc.RunningStats(first_step=first_step, threads=THREADS)
     for g, d in zip(g_list, d_list):
         n = g.numel()
@@ -52,11 +52,13 @@ def slices_of(n):
 def check_outputs_sampled(shapes, rho, config_id, g_dtype, g_gpu, d_gpu, hp, dec):
     ohp = to_orc_hp(hp)
     lim = 4 if g_dtype == torch.float32 else 1
+    d_dtype = d_gpu[0].dtype
     worst = 0
     for i in range(len(shapes)):
         (g0,), (d0,) = synth.gradient_list(shapes, rho, config_id, g_dtype, "cuda", indices=[i])
-        # state refresh: exact widening of the raw gradient, every element
-        assert torch.equal(d_gpu[i], g0.float()), f"tensor {i}: d' != raw g"
+        d0 = d0.to(d_dtype)
+        # state refresh: exact copy (or exact widening) of the raw gradient, every element
+        assert torch.equal(d_gpu[i], g0.to(d_dtype)), f"tensor {i}: d' != raw g"
         if dec.regime != orc.PROJECT:
             assert torch.equal(g_gpu[i], g0), f"tensor {i}: g changed outside the projection regime"
             continue
@@ -72,14 +74,77 @@ def check_outputs_sampled(shapes, rho, config_id, g_dtype, g_gpu, d_gpu, hp, dec
     return worst
 
 
+def test_config_fused_adamw_full_size():
+    """The projection fused with AdamW on the 7 B list (bf16 g, f32 d; 137 GB resident with p, m, v), in the
+    configuration bench.py times: one projection step with t = 6.  The oracle's sums run over every element;
+    p, m, v are compared on three slices of every tensor (whole tensors up to 32 M elements) with the bars of
+    the per-step test; d' = g is checked on every element and g must come out untouched."""
+    dims_key, g_dtype, rho, config_id = synth.WORKLOADS["cfg3_7b_bf16"]
+    shapes = synth.decoder_tensor_list(synth.DIMS[dims_key])
+    torch.cuda.empty_cache()
+    free, _ = torch.cuda.mem_get_info()
+    if free < (160 << 30):
+        pytest.skip(f"needs 160 GiB of device memory, {free >> 30} GiB free")
+    hp = gb.HParams(**FORCE)
+    ohp = to_orc_hp(hp)
+    gopt, oopt = gb.AdamW(lr=1e-4), orc.AdamW(lr=1e-4)
+
+    def state(i, n):
+        gen = torch.Generator(device="cuda").manual_seed(77_000 + i)
+        p = torch.randn(n, generator=gen, device="cuda") * 0.02
+        m = torch.randn(n, generator=gen, device="cuda") * 1e-3
+        v = torch.rand(n, generator=gen, device="cuda") * 1e-6
+        return p, m, v
+
+    g, d = synth.gradient_list(shapes, rho, config_id, g_dtype, "cuda")
+    p, m, v = (list(x) for x in zip(*(state(i, n) for i, (_, n) in enumerate(shapes))))
+    dec = orc.decide(oracle_sums_streamed(g, d), ohp)
+    assert dec.regime == orc.PROJECT
+    ctx = gb.gac_init(g, d, hp)
+    gb.gac_attach_adamw(ctx, p, m, v, applied_steps=5)
+    res = gb.gac_stats(ctx, 2)
+    after = gb.gac_project_adamw(ctx, gopt, coef_override=dec.coef, fetch=True)
+    torch.cuda.synchronize()
+    check_sums(res, dec)
+    check_decision(res, dec)
+    assert after.applied_steps == 6
+    gb.gac_free(ctx)
+    for i, (_, n) in enumerate(shapes):
+        (g0,), (d0,) = synth.gradient_list(shapes, rho, config_id, g_dtype, "cuda", indices=[i])
+        assert torch.equal(g[i].view(torch.int16), g0.view(torch.int16)), f"tensor {i}: g was written"
+        assert torch.equal(d[i], g0.float()), f"tensor {i}: d' != raw g"
+        p0, m0, v0 = state(i, n)
+        for lo, hi in slices_of(n):
+            ref = [x[lo:hi].cpu().contiguous() for x in (g0, d0, p0, m0, v0)]
+            m_before = ref[3].clone()
+            gmag = ref[0].float().abs() + abs(dec.coef) * ref[1].abs()
+            orc.project_adamw([ref[0]], [ref[1]], [ref[2]], [ref[3]], [ref[4]], ohp, dec, oopt, 6)
+            for name, got, want, slack in (("v", v[i], ref[4], None),
+                                           ("m", m[i], ref[3], 1e-13 * (m_before.abs() + gmag)),
+                                           ("p", p[i], ref[2], torch.full_like(ref[2], 1e-10 * oopt.lr))):
+                a = got[lo:hi].cpu()
+                ulps = (ordered_int(a) - ordered_int(want)).abs()
+                ok = ulps <= 4
+                if slack is not None:
+                    ok |= (a.double() - want.double()).abs() <= slack.double()
+                assert bool(ok.all()), f"tensor {i} [{lo}:{hi}] {name}: {int(ulps[~ok].max())} ulp"
+        del g0, d0, p0, m0, v0
+    del g, d, p, m, v
+    torch.cuda.empty_cache()
+
+
 def run_config(workload, hp):
     dims_key, g_dtype, rho, config_id = synth.WORKLOADS[workload]
+    d_dtype = synth.WORKLOAD_D_DTYPE.get(workload, torch.float32)
     shapes = synth.decoder_tensor_list(synth.DIMS[dims_key])
     need = synth.list_numel(shapes) * ((2 if g_dtype == torch.bfloat16 else 4) + 4) + (12 << 30)
+    torch.cuda.empty_cache()
     free, _ = torch.cuda.mem_get_info()
     if free < need:
         pytest.skip(f"needs {need >> 30} GiB of device memory, {free >> 30} GiB free")
     g, d = synth.gradient_list(shapes, rho, config_id, g_dtype, "cuda")
+    if d_dtype != torch.float32:
+        d = [t.to(d_dtype) for t in d]
     dec = orc.decide(oracle_sums_streamed(g, d), to_orc_hp(hp))
     ctx = gb.gac_init(g, d, hp)
     res = gb.gac_stats(ctx, 2, staleness=1)
@@ -97,7 +162,7 @@ def run_config(workload, hp):
     return res, dec, worst
 
 
-@pytest.mark.parametrize("workload", ["cfg2_1.5b_f32", "cfg3_7b_bf16", "cfg5_14b_f32"])
+@pytest.mark.parametrize("workload", ["cfg2_1.5b_f32", "cfg3_7b_bf16", "cfg5_14b_f32", "cfg3_7b_bf16_dbf16"])
 def test_config_projection_regime(workload):
     res, dec, worst = run_config(workload, gb.HParams(**FORCE))
     assert res.regime == gb.GAC_REGIME_PROJECT
