@@ -542,7 +542,7 @@ int gac_exchange_attach(gac_ctx *ctx, uint32_t rank, uint32_t world, void *const
     if (!slots) return fail(ctx, GAC_ERR_INVALID_ARG, "slots is NULL%s");
     if (ctx->stats_pending || ctx->decision_ready)
         return fail(ctx, GAC_ERR_STATE, "gac_exchange_attach between the calls of a step would split it%s");
-    std::vector<unsigned long long> table(world);
+    unsigned long long table[GAC_EXCHANGE_MAX_RANKS];   // on the stack: this call must not throw
     for (uint32_t r = 0; r < world; ++r) {
         const uint64_t a = reinterpret_cast<uint64_t>(slots[r]);
         if (!a || a % sizeof(PeerSlot))
@@ -555,7 +555,7 @@ int gac_exchange_attach(gac_ctx *ctx, uint32_t rank, uint32_t world, void *const
         ctx->d_peers = nullptr;
     }
     GAC_CUDA(ctx, cudaMalloc(&ctx->d_peers, world * sizeof(unsigned long long)));
-    GAC_CUDA(ctx, cudaMemcpy(ctx->d_peers, table.data(), world * sizeof(unsigned long long), cudaMemcpyHostToDevice));
+    GAC_CUDA(ctx, cudaMemcpy(ctx->d_peers, table, world * sizeof(unsigned long long), cudaMemcpyHostToDevice));
     ctx->xchg_world = world;
     ctx->xchg_rank = rank;
     ctx->xchg_slots = static_cast<PeerSlot *>(slots[rank]);
