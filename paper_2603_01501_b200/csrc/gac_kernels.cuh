@@ -31,9 +31,6 @@ namespace {
 #ifndef GAC_PHASE_BARRIER   // 1: the fused AdamW pass keeps the warps of a CTA in step (see phase_barrier)
 #define GAC_PHASE_BARRIER 1
 #endif
-#ifndef GAC_PROJECT_BARRIER   // the same in the projection pass: bit 0 after the loads, bit 1 after the stores
-#define GAC_PROJECT_BARRIER 1   // after the loads: +0.5-1 % on B200; after the stores it costs 2-10 % there
-#endif
 constexpr int kDefaultChunk = GAC_CHUNK; // elements per chunk
 constexpr int kMaxCtasPerSm = 16;
 
@@ -161,6 +158,8 @@ using DOf = typename PairOf<P>::D;
 //   UK    the same for a step that leaves g alone (only g read, only d written)
 //   C     resident CTAs per SM the grid is sized for (0 = all that fit)
 //   MINB  occupancy asked of the compiler through __launch_bounds__
+//   BAR   projection: __syncthreads() after a batch's loads (bit 0) and/or after its stores (bit 1)
+//   PF    projection: 1 = the next chunk's descriptor is fetched while the current chunk is worked on
 // A build that times variants substitutes its own table with
 // -DGAC_GEOMETRY_HEADER='"file.h"'.
 template <typename P>
@@ -177,12 +176,12 @@ struct AdamGeom;    // projection fused with AdamW
 template <> struct StatsGeom<float>       { static constexpr int T = 256, U = 8, C = 0, MINB = 4; };
 template <> struct StatsGeom<bf16_t>      { static constexpr int T = 256, U = 8, C = 0, MINB = 4; };
 template <> struct StatsGeom<bf16_pair_t> { static constexpr int T = 256, U = 8, C = 0, MINB = 4; };
-template <> struct ProjGeom<float>        { static constexpr int T = 256, U = 8, UK = 16, C = 1, MINB = 1; };
-template <> struct ProjGeom<bf16_t>       { static constexpr int T = 512, U = 4, UK = 8, C = 1, MINB = 1; };
-template <> struct ProjGeom<bf16_pair_t>  { static constexpr int T = 512, U = 8, UK = 8, C = 1, MINB = 1; };
-template <> struct ExchGeom<float>        { static constexpr int T = 512, U = 4, UK = 8, C = 1, MINB = 1; };
-template <> struct ExchGeom<bf16_t>       { static constexpr int T = 512, U = 4, UK = 8, C = 1, MINB = 1; };   // pair not served
-template <> struct ExchGeom<bf16_pair_t>  { static constexpr int T = 512, U = 4, UK = 8, C = 2, MINB = 2; };
+template <> struct ProjGeom<float>        { static constexpr int T = 256, U = 8, UK = 16, C = 1, MINB = 1, BAR = 2, PF = 1; };
+template <> struct ProjGeom<bf16_t>       { static constexpr int T = 512, U = 4, UK = 8, C = 1, MINB = 1, BAR = 1, PF = 1; };
+template <> struct ProjGeom<bf16_pair_t>  { static constexpr int T = 512, U = 8, UK = 8, C = 1, MINB = 1, BAR = 1, PF = 0; };
+template <> struct ExchGeom<float>        { static constexpr int T = 512, U = 4, UK = 8, C = 1, MINB = 1, BAR = 1, PF = 0; };
+template <> struct ExchGeom<bf16_t>       { static constexpr int T = 512, U = 4, UK = 8, C = 1, MINB = 1, BAR = 1, PF = 0; };   // pair not served
+template <> struct ExchGeom<bf16_pair_t>  { static constexpr int T = 512, U = 4, UK = 8, C = 2, MINB = 2, BAR = 1, PF = 0; };
 // AdamGeom: T threads for the plain rule (beta = 1, no clipping), TG for the general one, C CTAs per SM.
 // float32 gradients: one CTA of 1024 threads (a 64 KB chunk is exactly four batches); bfloat16
 // gradients move fewer bytes per batch, and two CTAs of 512 threads, each in step with itself
@@ -603,7 +602,7 @@ __device__ __forceinline__ float rank_one(float g, float d, float k, double beta
 }
 __device__ __forceinline__ float scaled(float g, double s) { return __double2float_rn(__dmul_rn(s, double(g))); }
 
-template <typename GT, int GOP, int DOP, bool BETA1, int T, int U>
+template <typename GT, int GOP, int DOP, bool BETA1, int T, int U, int BAR>
 __device__ __forceinline__ void project_chunk(const Chunk &ch, float k, double beta, double s) {
     void *g = reinterpret_cast<void *>(ch.g);
     void *d = reinterpret_cast<void *>(ch.d);
@@ -626,7 +625,7 @@ __device__ __forceinline__ void project_chunk(const Chunk &ch, float k, double b
                     if (kReadD) dr[u] = Elem<DOf<GT>>::template load_raw<GAC_LD_PROJECT>(d, v);
                 }
             }
-            if (GAC_PROJECT_BARRIER & 1) __syncthreads();
+            if (BAR & 1) __syncthreads();   // keeps the warps of the CTA in step (see phase_barrier)
 #pragma unroll
             for (int u = 0; u < U; ++u) {
                 const uint32_t v = base + u * T + tid;
@@ -649,7 +648,7 @@ __device__ __forceinline__ void project_chunk(const Chunk &ch, float k, double b
                     Elem<DOf<GT>>::store4(d, v, out);
                 }
             }
-            if (GAC_PROJECT_BARRIER & 2) __syncthreads();
+            if (BAR & 2) __syncthreads();
         }
         const uint32_t done = nvec << 2;
         if (tid < ch.n - done) {
@@ -685,21 +684,60 @@ __device__ __forceinline__ void project_chunk(const Chunk &ch, float k, double b
 template <typename GT, int STATE>
 using ProjGeomOf = typename std::conditional<STATE == GAC_STATE_EXCHANGE, ExchGeom<GT>, ProjGeom<GT>>::type;
 
-// A CTA's walk over its chunks.  Every thread reads the descriptor when it gets to the chunk: the
-// short wait for it lets the warps of the CTA fall into step again at every chunk boundary, which
-// this pass likes (fetching the descriptor ahead of time, through registers or asynchronously
-// through shared memory, measured no better for f32 and 2-5 % worse for bfloat16 gradients).
-template <typename GT, int GOP, int DOP, bool BETA1, int T, int U>
+// The descriptor of chunk c, read with loads the compiler may not move: a prefetch only helps if it
+// is issued where it is written, ahead of the chunk's work.
+__device__ __forceinline__ void load_chunk_words(const Chunk *table, uint32_t c, uint4 &a, uint4 &b) {
+    const uint4 *p = reinterpret_cast<const uint4 *>(table + c);
+    asm volatile("ld.global.nc.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(a.x), "=r"(a.y), "=r"(a.z), "=r"(a.w) : "l"(p));
+    asm volatile("ld.global.nc.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(b.x), "=r"(b.y), "=r"(b.z), "=r"(b.w) : "l"(p + 1));
+}
+__device__ __forceinline__ Chunk chunk_from_words(uint4 a, uint4 b, int swapped) {
+    Chunk ch;
+    ch.g = (uint64_t(a.y) << 32) | a.x;
+    ch.d = (uint64_t(a.w) << 32) | a.z;
+    if (swapped) {
+        const uint64_t t = ch.g;
+        ch.g = ch.d;
+        ch.d = t;
+    }
+    ch.n = b.x;
+    ch.flags = b.y;
+    ch.pad = 0;
+    return ch;
+}
+
+// A CTA's walk over its chunks.  How the warps of the CTA line up decides how well DRAM is used
+// (see phase_barrier), and two arrangements work on B200:
+//   PF = 0  every thread reads the descriptor when it gets to the chunk; the short wait for it lets
+//           the warps fall into step again at every chunk boundary (with BAR = 1 on top: +0.5-1 %);
+//   PF = 1  the next descriptor is fetched while the current chunk is worked on, and barriers alone
+//           keep the warps in step.  With BAR = 2 this is the fastest form for float32 pairs
+//           (6.67 against 6.54 TB/s on the 1.5 B list) and the slowest for bfloat16 gradients; with
+//           BAR = 1 it leaves the projection of bf16/f32 lists as it was and speeds up their steps
+//           that only refresh the stored direction by 2 %.
+template <typename GT, int GOP, int DOP, bool BETA1, int T, int U, int PF, int BAR>
 __device__ __forceinline__ void project_walk_tu(const Chunk *chunks, uint32_t n_chunks, float k,
                                                 double beta, double s, int swapped) {
-    for (uint32_t c = blockIdx.x; c < n_chunks; c += gridDim.x)
-        project_chunk<GT, GOP, DOP, BETA1, T, U>(load_chunk(chunks, c, swapped), k, beta, s);
+    if (PF) {
+        uint32_t c = blockIdx.x;
+        if (c >= n_chunks) return;
+        uint4 wa, wb;
+        load_chunk_words(chunks, c, wa, wb);
+        for (; c < n_chunks; c += gridDim.x) {
+            const Chunk ch = chunk_from_words(wa, wb, swapped);
+            if (c + gridDim.x < n_chunks) load_chunk_words(chunks, c + gridDim.x, wa, wb);
+            project_chunk<GT, GOP, DOP, BETA1, T, U, BAR>(ch, k, beta, s);
+        }
+    } else {
+        for (uint32_t c = blockIdx.x; c < n_chunks; c += gridDim.x)
+            project_chunk<GT, GOP, DOP, BETA1, T, U, BAR>(load_chunk(chunks, c, swapped), k, beta, s);
+    }
 }
 template <typename GT, int GOP, int DOP, bool BETA1>
 __device__ __forceinline__ void project_walk(const Chunk *chunks, uint32_t n_chunks, float k,
                                              double beta, double s, int swapped) {
     using Geom = typename std::conditional<DOP == D_OUT, ExchGeom<GT>, ProjGeom<GT>>::type;
-    project_walk_tu<GT, GOP, DOP, BETA1, Geom::T, Geom::U>(chunks, n_chunks, k, beta, s, swapped);
+    project_walk_tu<GT, GOP, DOP, BETA1, Geom::T, Geom::U, Geom::PF, Geom::BAR>(chunks, n_chunks, k, beta, s, swapped);
 }
 
 // The regime is read from the device-resident record, so no host round trip
@@ -740,7 +778,8 @@ gac_project_kernel(const Chunk *__restrict__ chunks, uint32_t n_chunks, gac_resu
         project_walk<GT, G_SCALE, dop, true>(chunks, n_chunks, k, 1.0, s, swapped);   // safe step, clipped: g'' = s g
     } else if (STATE != GAC_STATE_HOLD && STATE != GAC_STATE_EXCHANGE) {
         // d' = g, g untouched
-        project_walk_tu<GT, G_KEEP, D_RAW, true, ProjGeom<GT>::T, ProjGeom<GT>::UK>(chunks, n_chunks, k, 1.0, 1.0, 0);
+        project_walk_tu<GT, G_KEEP, D_RAW, true, ProjGeom<GT>::T, ProjGeom<GT>::UK, ProjGeom<GT>::PF, ProjGeom<GT>::BAR>(
+            chunks, n_chunks, k, 1.0, 1.0, 0);
     }
     // exchange mode, g unchanged: nothing to move -- the buffers that hold g become the stored direction
 }
@@ -985,7 +1024,7 @@ gac_adamw_kernel(const Chunk *__restrict__ chunks, const OptChunk *__restrict__ 
         else if (!PLAIN) adamw_walk<GT, G_SCALE, !EXCH, T>(chunks, opt_chunks, n_chunks, swapped, 1.0, s, o, st);
     } else if (!EXCH) {
         // skipped step: d' = g only
-        project_walk_tu<GT, G_KEEP, D_RAW, true, AdamThreads<GT, PLAIN>::T, AdamGeom<GT>::U>(chunks, n_chunks, k, 1.0, 1.0, 0);
+        project_walk_tu<GT, G_KEEP, D_RAW, true, AdamThreads<GT, PLAIN>::T, AdamGeom<GT>::U, 0, 1>(chunks, n_chunks, k, 1.0, 1.0, 0);
     }
     __syncthreads();
     if (threadIdx.x == 0) {
